@@ -11,6 +11,7 @@ Nothing here quantizes, dithers, packs or decodes anything.
 """
 from __future__ import annotations
 
+import functools
 from dataclasses import dataclass, field
 from typing import Callable, List, Optional
 
@@ -79,6 +80,7 @@ def tiny(n: int = 65536, W: int = 2, bucket: int = 512, seed: int = 0, bits: int
     kind: "dqsg" (all workers b-bit DQSG), "ndqsg" (all NDQSG, K = M1 = 2^b), or
     "mixed" (worker 0 DQSG, the rest NDQSG).
     """
+    @functools.lru_cache(maxsize=1)
     def common():
         return (0.1 * _normal32(_rng(seed, 1), n)).astype(np.float32)
 
@@ -133,6 +135,7 @@ def ndqsg_resnet50(n: int = 25_557_032, W: int = 8, bucket: int = 2048, seed: in
     """c ~ N(0,1e-4), n_w ~ N(0,1e-4), g_w = c + n_w/3 (pairwise correlation 0.9).
     Worker 0: DQSG with L=5 (M=2, Delta=0.5, 3 bits); workers 1..W-1: NDQSG K=4 (2 bits), M1=2, alpha=1.
     Side information for the NDQSG workers is worker 0's decoded gradient."""
+    @functools.lru_cache(maxsize=1)
     def common():
         return (np.float32(1e-2) * _normal32(_rng(seed, 6), n)).astype(np.float32)
 
@@ -151,6 +154,7 @@ def ndqsg_resnet50(n: int = 25_557_032, W: int = 8, bucket: int = 2048, seed: in
 # --------------------------------------------------------------------------
 def ndqsg_gpt2_small(n: int = 124_439_808, W: int = 16, bucket: int = 4096, seed: int = 0) -> Workload:
     """c ~ Laplace(0,1e-3); g_w = c + N(0,(3e-4)^2); y = c + N(0,(1e-4)^2); all NDQSG K=8 (3 bits), M1=16."""
+    @functools.lru_cache(maxsize=1)
     def common():
         r = _rng(seed, 8)
         out = np.empty(n, dtype=np.float32)

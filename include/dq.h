@@ -1,0 +1,159 @@
+/*
+ * dq.h -- C ABI of the dithered / nested dithered gradient quantizer for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-worker encoder and the server-side decode-and-average step of
+ * Abdi & Fekri, "Nested Dithered Quantization for Communication Reduction in Distributed Training":
+ *
+ *   DQSG   (Section 3.1, Eq. (DQSG), Algorithm 1):  g~ = kappa (Q(g/kappa + u) - u),  kappa = ||g||_inf,
+ *          u ~ U[-Delta/2, Delta/2] regenerated at the receiver from a shared seed; the worker sends
+ *          kappa and the bin index.
+ *   NDQSG  (Section 3.2, nested encoder / decoder equations, Algorithm 2):  t = alpha g + u,
+ *          s = Q1(t) - Q2(t);  r = s - u - alpha y,  g^ = y + alpha (r - Q2(r))  with side information y.
+ *
+ * Conventions shared by every entry point
+ *   - A gradient is a flat fp32 vector of n elements, cut into buckets of `bucket` elements (the paper's
+ *     equal partitions, one scale kappa each; the last bucket may be short).
+ *   - The dither of element i of worker `worker` at iteration `step` is word (i mod 4) of
+ *     Philox4x32-10(key = seed, counter = (i / 4, worker, lo32(step), hi32(step))), mapped to the open
+ *     grid {(2j+1) 2^-23 - 1/2} in units of the fine quantization step.  Encoder and decoder must be
+ *     given the same (seed, worker, step).
+ *   - A message is `scale` (one fp32 per bucket) plus `packed`: element i's b-bit code at bit offset
+ *     i*b of a little-endian stream of 32-bit words; pad bits of the last word are written as 0.
+ *   - "device" pointers are CUDA device memory on the current device, 16-byte aligned, owned by the
+ *     caller.  The library allocates nothing, keeps no state between calls, and is asynchronous on the
+ *     given stream (it never synchronises), except for the *_host entry points, which return after the
+ *     results are in the caller's host buffers.
+ *   - Outputs must not alias inputs.  Inputs are assumed finite.
+ *   - Errors are return codes only.  Invalid arguments are rejected before anything is launched.
+ *   - n must be below 2^34.
+ */
+#ifndef DQ_H_
+#define DQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DQ_OK = 0,
+    DQ_ERR_INVALID_ARG = 1,   /* NULL pointer, n or W out of range, bits/levels/K/alpha out of range      */
+    DQ_ERR_UNSUPPORTED = 2,   /* valid in the paper's terms but not handled (e.g. mixed bucket sizes)     */
+    DQ_ERR_ALIGNMENT = 3,     /* a device pointer is not 16-byte aligned                                  */
+    DQ_ERR_CUDA = 4           /* a CUDA call or launch failed; see cudaGetLastError of the calling thread */
+} dq_status;
+
+typedef enum { DQ_KIND_DQSG = 0, DQ_KIND_NDQSG = 1 } dq_kind;
+
+/* Bits of the optional decode status word and of dq_device_error_flags(). */
+#define DQ_WARN_NONFINITE_SCALE 0x1u   /* a received scale was NaN or Inf                                   */
+#define DQ_ERR_COPY_TIMEOUT     0x2u   /* a bounded wait for an asynchronous tile copy ran out; the tile
+                                          was skipped and its outputs are undefined                        */
+
+/* One quantizer description.  Plain data, read during the call. */
+typedef struct {
+    uint32_t bucket;    /* B: multiple of 32 in [32, 65536]                                               */
+    uint32_t bits;      /* b: 1..8 bits per element on the wire                                           */
+    uint32_t levels;    /* DQSG: number of levels L, 2..2^b (odd L = the paper's 2M+1, Delta = 2/(L-1));
+                           0 selects L = 2 for b = 1 and 2^b - 1 otherwise.  Ignored for NDQSG.           */
+    uint32_t coarse_K;  /* NDQSG: K = Delta_2 / Delta_1, 2..2^b.  Ignored for DQSG.                       */
+    float    fine_M;    /* NDQSG: M1 = 1/Delta_1 in units of kappa, 0 < alpha*M1 <= 2^20.                 */
+    float    alpha;     /* NDQSG: shrinkage, 0 < alpha <= 1; 0 selects 1.                                 */
+} dq_params;
+
+/* One worker's message as the decoder sees it. */
+typedef struct {
+    const uint32_t* packed;  /* dq_packed_words(n, p.bits) words                                          */
+    const float*    scale;   /* dq_num_buckets(n, p.bucket) scales                                        */
+    uint64_t        seed;    /* the worker's dither seed                                                  */
+    uint32_t        worker;  /* the worker's index as used by its encoder                                 */
+    dq_kind         kind;
+    dq_params       p;
+} dq_msg;
+
+#define DQ_MAX_WORKERS 64u
+
+/* Message sizes: ceil(n*bits/32) words and ceil(n/bucket) scales. */
+uint64_t dq_packed_words(uint64_t n, uint32_t bits);
+uint64_t dq_num_buckets(uint64_t n, uint32_t bucket);
+/* The level count used when dq_params.levels is 0. */
+uint32_t dq_default_levels(uint32_t bits);
+const char* dq_status_string(dq_status s);
+
+/*
+ * dqsg_encode -- worker side of Algorithm 1 (Eq. (DQSG)): per bucket kappa = max|g|, dither from
+ * (seed, worker, step), index q = round((g/kappa + u)/Delta) stored as k = q + (L-1)/2 in b bits.
+ *   grad        device, fp32[n], read once
+ *   out_packed  device, uint32[dq_packed_words(n, p->bits)], fully overwritten
+ *   out_scale   device, fp32[dq_num_buckets(n, p->bucket)], fully overwritten
+ *   cuda_stream a cudaStream_t (NULL = default stream)
+ * n = 0 is a no-op returning DQ_OK.
+ */
+dq_status dqsg_encode(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                      const dq_params* p, uint32_t* out_packed, float* out_scale, void* cuda_stream);
+
+/*
+ * ndqsg_encode -- worker side of Algorithm 2 for a worker in P2 (nested encoder equation), with the
+ * per-bucket normalisation of Algorithm 1: q1 = round(alpha*M1*g/kappa + u/Delta_1), and the message is
+ * the coset q1 mod K in [0, K), which determines s = Q1(t) - Q2(t).  Same buffers as dqsg_encode.
+ */
+dq_status ndqsg_encode(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                       const dq_params* p, uint32_t* out_packed, float* out_scale, void* cuda_stream);
+
+/*
+ * dqsg_decode_aggregate -- server side of Algorithm 1: regenerate every worker's dither, reconstruct
+ * g~_w = kappa_w (Delta q_w - u_w) and write the mean over the W workers, summed in array order.
+ *   msgs     host array of W messages (1 <= W <= DQ_MAX_WORKERS), all of kind DQSG and of one bucket
+ *            size; read during the call, the device buffers they point to are read by the kernel
+ *   out_avg  device, fp32[n], fully overwritten
+ */
+dq_status dqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                float* out_avg, void* cuda_stream);
+
+/*
+ * ndqsg_decode_aggregate -- server side of Algorithm 2 with the side information given as a vector
+ * (nested decoder equation): DQSG messages are reconstructed as above; an NDQSG message is resolved to
+ * the fine index congruent to its code that lies in the coarse cell around alpha*M1*y/kappa, and
+ * reconstructed as g^ = (1 - alpha^2) y + (alpha kappa / M1)(q1^ - u/Delta_1); the mean of all W
+ * reconstructions is written.  Kinds, bits, levels, K, M1 and alpha may differ per worker.
+ *   side_info    device, fp32[n]; required when any message is NDQSG, may be NULL otherwise
+ *   status_word  device uint32, optional (NULL to skip): DQ_WARN_* bits are OR-ed into it
+ */
+dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                 const float* side_info, float* out_avg, uint32_t* status_word,
+                                 void* cuda_stream);
+
+/*
+ * Host-buffer variants.  Every data pointer (grad, out_packed, out_scale, the packed/scale pointers
+ * inside msgs, side_info, out_avg) is HOST memory (pinned memory makes the copies asynchronous);
+ * `workspace` is device memory of at least the stated size, 256-byte aligned, provided by the caller.
+ * Each call copies its inputs to the workspace, runs the same kernels as the device entry points,
+ * copies the results back and synchronises the stream before returning.
+ */
+uint64_t dq_encode_workspace_bytes(uint64_t n, const dq_params* p);
+uint64_t dq_decode_workspace_bytes(const dq_msg* msgs, uint32_t W, uint64_t n, int has_side_info);
+dq_status dqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                           const dq_params* p, uint32_t* out_packed, float* out_scale,
+                           void* workspace, uint64_t workspace_bytes, void* cuda_stream);
+dq_status ndqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                            const dq_params* p, uint32_t* out_packed, float* out_scale,
+                            void* workspace, uint64_t workspace_bytes, void* cuda_stream);
+dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                      const float* side_info, float* out_avg,
+                                      void* workspace, uint64_t workspace_bytes, void* cuda_stream);
+
+/*
+ * dq_device_error_flags -- reads (and clears) the current device's error word: DQ_ERR_COPY_TIMEOUT is
+ * set if any kernel of this library gave up waiting for one of its own asynchronous copies.
+ * Synchronises the device.
+ */
+dq_status dq_device_error_flags(uint32_t* out_flags);
+
+/* Number of kernel launches issued by this library in the calling process so far. */
+uint64_t dq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DQ_H_ */

@@ -1,0 +1,249 @@
+"""ctypes binding of ``libdq_b200.so``.  Argument marshalling only.
+
+Tensors are ``torch`` CUDA tensors (device entry points) or CPU tensors / numpy arrays (``*_host`` entry
+points); the binding passes their addresses and the current CUDA stream to the C ABI and raises
+``DqError`` on a non-zero status.  There is no fallback: if the shared library is missing the import of
+``lib()`` fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+from typing import Optional, Sequence
+
+import torch
+
+DQ_KIND_DQSG = 0
+DQ_KIND_NDQSG = 1
+DQ_WARN_NONFINITE_SCALE = 0x1
+DQ_ERR_COPY_TIMEOUT = 0x2
+
+_LIB_PATH = Path(__file__).resolve().parent / "lib" / "libdq_b200.so"
+
+
+class DqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (status {status})")
+
+
+class DqParams(C.Structure):
+    _fields_ = [("bucket", C.c_uint32), ("bits", C.c_uint32), ("levels", C.c_uint32),
+                ("coarse_K", C.c_uint32), ("fine_M", C.c_float), ("alpha", C.c_float)]
+
+
+class DqMsg(C.Structure):
+    _fields_ = [("packed", C.c_void_p), ("scale", C.c_void_p), ("seed", C.c_uint64),
+                ("worker", C.c_uint32), ("kind", C.c_int), ("p", DqParams)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads the CUDA library (built by ``paper_1904_01197_b200.build``).  Fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_1904_01197_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(str(_LIB_PATH))
+        vp, u64, u32 = C.c_void_p, C.c_uint64, C.c_uint32
+        pp = C.POINTER(DqParams)
+        pm = C.POINTER(DqMsg)
+        L.dq_packed_words.argtypes = [u64, u32]; L.dq_packed_words.restype = u64
+        L.dq_num_buckets.argtypes = [u64, u32]; L.dq_num_buckets.restype = u64
+        L.dq_default_levels.argtypes = [u32]; L.dq_default_levels.restype = u32
+        L.dq_status_string.argtypes = [C.c_int]; L.dq_status_string.restype = C.c_char_p
+        for f in (L.dqsg_encode, L.ndqsg_encode):
+            f.argtypes = [vp, u64, u64, u32, u64, pp, vp, vp, vp]; f.restype = C.c_int
+        L.dqsg_decode_aggregate.argtypes = [pm, u32, u64, u64, vp, vp]
+        L.dqsg_decode_aggregate.restype = C.c_int
+        L.ndqsg_decode_aggregate.argtypes = [pm, u32, u64, u64, vp, vp, vp, vp]
+        L.ndqsg_decode_aggregate.restype = C.c_int
+        L.dq_encode_workspace_bytes.argtypes = [u64, pp]; L.dq_encode_workspace_bytes.restype = u64
+        L.dq_decode_workspace_bytes.argtypes = [pm, u32, u64, C.c_int]; L.dq_decode_workspace_bytes.restype = u64
+        for f in (L.dqsg_encode_host, L.ndqsg_encode_host):
+            f.argtypes = [vp, u64, u64, u32, u64, pp, vp, vp, vp, u64, vp]; f.restype = C.c_int
+        L.ndqsg_decode_aggregate_host.argtypes = [pm, u32, u64, u64, vp, vp, vp, u64, vp]
+        L.ndqsg_decode_aggregate_host.restype = C.c_int
+        L.dq_device_error_flags.argtypes = [C.POINTER(u32)]; L.dq_device_error_flags.restype = C.c_int
+        L.dq_launch_count.argtypes = []; L.dq_launch_count.restype = u64
+        _lib = L
+    return _lib
+
+
+def packed_words(n: int, bits: int) -> int:
+    return int(lib().dq_packed_words(n, bits))
+
+
+def num_buckets(n: int, bucket: int) -> int:
+    return int(lib().dq_num_buckets(n, bucket))
+
+
+def default_levels(bits: int) -> int:
+    return int(lib().dq_default_levels(bits))
+
+
+def status_string(status: int) -> str:
+    return lib().dq_status_string(status).decode()
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise DqError(status, what)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype, what: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{what}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _host_ptr(t, dtype, what: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor):
+        t = torch.from_numpy(t)
+    if t.is_cuda or not t.is_contiguous() or t.dtype != dtype:
+        raise TypeError(f"{what}: expected a contiguous CPU tensor of {dtype}")
+    return t.data_ptr()
+
+
+def make_params(bucket: int, bits: int, levels: int = 0, coarse_K: int = 0, fine_M: float = 0.0,
+                alpha: float = 0.0) -> DqParams:
+    return DqParams(bucket, bits, levels, coarse_K, fine_M, alpha)
+
+
+class Message:
+    """A worker's message on the device plus what the decoder must know about it."""
+
+    def __init__(self, packed: torch.Tensor, scale: torch.Tensor, seed: int, worker: int, kind: int,
+                 params: DqParams):
+        self.packed, self.scale = packed, scale
+        self.seed, self.worker, self.kind, self.params = seed, worker, kind, params
+
+    def as_struct(self, host: bool = False) -> DqMsg:
+        if host:
+            pk = _host_ptr(self.packed, torch.int32, "packed")
+            sc = _host_ptr(self.scale, torch.float32, "scale")
+        else:
+            pk = _dev_ptr(self.packed, torch.int32, "packed")
+            sc = _dev_ptr(self.scale, torch.float32, "scale")
+        return DqMsg(pk, sc, self.seed, self.worker, self.kind, self.params)
+
+
+def alloc_message(n: int, params: DqParams, device="cuda"):
+    """Uninitialised output buffers for one encode call (packed words as int32, scales as fp32)."""
+    packed = torch.empty(max(1, packed_words(n, params.bits)), dtype=torch.int32, device=device)
+    scale = torch.empty(max(1, num_buckets(n, params.bucket)), dtype=torch.float32, device=device)
+    return packed, scale
+
+
+def _encode(fn, what, grad, seed, worker, step, params, out_packed, out_scale, stream):
+    n = grad.numel()
+    if out_packed is None or out_scale is None:
+        out_packed, out_scale = alloc_message(n, params, grad.device)
+    if out_packed.numel() < packed_words(n, params.bits) or out_scale.numel() < num_buckets(n, params.bucket):
+        raise ValueError(f"{what}: output buffers too small")
+    _check(fn(_dev_ptr(grad, torch.float32, "grad"), n, seed, worker, step, C.byref(params),
+              _dev_ptr(out_packed, torch.int32, "out_packed"), _dev_ptr(out_scale, torch.float32, "out_scale"),
+              _stream_ptr(stream)), what)
+    return out_packed, out_scale
+
+
+def dqsg_encode(grad: torch.Tensor, seed: int, worker: int, step: int, params: DqParams,
+                out_packed: Optional[torch.Tensor] = None, out_scale: Optional[torch.Tensor] = None,
+                stream=None):
+    return _encode(lib().dqsg_encode, "dqsg_encode", grad, seed, worker, step, params, out_packed, out_scale, stream)
+
+
+def ndqsg_encode(grad: torch.Tensor, seed: int, worker: int, step: int, params: DqParams,
+                 out_packed: Optional[torch.Tensor] = None, out_scale: Optional[torch.Tensor] = None,
+                 stream=None):
+    return _encode(lib().ndqsg_encode, "ndqsg_encode", grad, seed, worker, step, params, out_packed, out_scale, stream)
+
+
+def _msg_array(msgs: Sequence[Message], host: bool = False):
+    arr = (DqMsg * max(1, len(msgs)))()
+    for i, m in enumerate(msgs):
+        arr[i] = m.as_struct(host)
+    return arr
+
+
+def dqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, out_avg: Optional[torch.Tensor] = None,
+                          stream=None) -> torch.Tensor:
+    if out_avg is None:
+        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+    _check(lib().dqsg_decode_aggregate(_msg_array(msgs), len(msgs), n, step,
+                                       _dev_ptr(out_avg, torch.float32, "out_avg"), _stream_ptr(stream)),
+           "dqsg_decode_aggregate")
+    return out_avg
+
+
+def ndqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, side_info: Optional[torch.Tensor],
+                           out_avg: Optional[torch.Tensor] = None, status_word: Optional[torch.Tensor] = None,
+                           stream=None) -> torch.Tensor:
+    if out_avg is None:
+        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+    _check(lib().ndqsg_decode_aggregate(_msg_array(msgs), len(msgs), n, step,
+                                        _dev_ptr(side_info, torch.float32, "side_info"),
+                                        _dev_ptr(out_avg, torch.float32, "out_avg"),
+                                        _dev_ptr(status_word, torch.int32, "status_word"), _stream_ptr(stream)),
+           "ndqsg_decode_aggregate")
+    return out_avg
+
+
+# ------------------------------------------------------------------------------------------ host buffers
+def encode_workspace_bytes(n: int, params: DqParams) -> int:
+    return int(lib().dq_encode_workspace_bytes(n, C.byref(params)))
+
+
+def decode_workspace_bytes(msgs: Sequence[Message], n: int, has_side_info: bool) -> int:
+    return int(lib().dq_decode_workspace_bytes(_msg_array(msgs, host=True), len(msgs), n, int(has_side_info)))
+
+
+def _encode_host(fn, what, grad, seed, worker, step, params, out_packed, out_scale, workspace, stream):
+    n = grad.numel()
+    _check(fn(_host_ptr(grad, torch.float32, "grad"), n, seed, worker, step, C.byref(params),
+              _host_ptr(out_packed, torch.int32, "out_packed"), _host_ptr(out_scale, torch.float32, "out_scale"),
+              workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream)), what)
+    return out_packed, out_scale
+
+
+def dqsg_encode_host(grad, seed, worker, step, params, out_packed, out_scale, workspace, stream=None):
+    return _encode_host(lib().dqsg_encode_host, "dqsg_encode_host", grad, seed, worker, step, params,
+                        out_packed, out_scale, workspace, stream)
+
+
+def ndqsg_encode_host(grad, seed, worker, step, params, out_packed, out_scale, workspace, stream=None):
+    return _encode_host(lib().ndqsg_encode_host, "ndqsg_encode_host", grad, seed, worker, step, params,
+                        out_packed, out_scale, workspace, stream)
+
+
+def ndqsg_decode_aggregate_host(msgs: Sequence[Message], n: int, step: int, side_info, out_avg, workspace,
+                                stream=None):
+    _check(lib().ndqsg_decode_aggregate_host(_msg_array(msgs, host=True), len(msgs), n, step,
+                                             _host_ptr(side_info, torch.float32, "side_info"),
+                                             _host_ptr(out_avg, torch.float32, "out_avg"),
+                                             workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                             _stream_ptr(stream)), "ndqsg_decode_aggregate_host")
+    return out_avg
+
+
+def device_error_flags() -> int:
+    v = C.c_uint32(0)
+    _check(lib().dq_device_error_flags(C.byref(v)), "dq_device_error_flags")
+    return int(v.value)
+
+
+def launch_count() -> int:
+    return int(lib().dq_launch_count())

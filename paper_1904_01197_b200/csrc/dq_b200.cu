@@ -1,0 +1,459 @@
+// Host side of the C ABI declared in include/dq.h: argument checks, tensor-map set-up, kernel launches.
+// Everything numerical happens in the kernels of dq_encode.cuh / dq_decode.cuh.
+#include "dq.h"
+
+#include <atomic>
+#include <cstring>
+
+#include "dq_decode.cuh"
+#include "dq_encode.cuh"
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+
+bool is_pow2(uint32_t v) { return v && !(v & (v - 1u)); }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0u; }
+
+void fill_philox(dq::PhiloxStream& ps, uint64_t seed, uint32_t worker, uint64_t step)
+{
+    uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFull), k1 = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        ps.rk[r][0] = k0;
+        ps.rk[r][1] = k1;
+        k0 += dq::kPhiloxW0;
+        k1 += dq::kPhiloxW1;
+    }
+    ps.c1 = worker;
+    ps.c2 = (uint32_t)(step & 0xFFFFFFFFull);
+    ps.c3 = (uint32_t)(step >> 32);
+}
+
+dq_status check_params(const dq_params* p, dq_kind kind, uint32_t* levels_out, float* alpha_out)
+{
+    if (!p) return DQ_ERR_INVALID_ARG;
+    if (p->bucket < 32u || p->bucket > 65536u || (p->bucket % 32u) != 0u) return DQ_ERR_INVALID_ARG;
+    if (p->bits < 1u || p->bits > 8u) return DQ_ERR_INVALID_ARG;
+    if (kind == DQ_KIND_DQSG) {
+        const uint32_t L = p->levels ? p->levels : dq_default_levels(p->bits);
+        if (L < 2u || L > (1u << p->bits)) return DQ_ERR_INVALID_ARG;
+        *levels_out = L;
+        *alpha_out = 1.0f;
+    } else if (kind == DQ_KIND_NDQSG) {
+        const float alpha = (p->alpha == 0.0f) ? 1.0f : p->alpha;
+        if (p->coarse_K < 2u || p->coarse_K > (1u << p->bits)) return DQ_ERR_INVALID_ARG;
+        if (!(p->fine_M > 0.0f) || !(alpha > 0.0f) || alpha > 1.0f) return DQ_ERR_INVALID_ARG;
+        const float A = alpha * p->fine_M;
+        if (!(A > 0.0f)) return DQ_ERR_INVALID_ARG;
+        if (A > 1048576.0f) return DQ_ERR_UNSUPPORTED;
+        *levels_out = 0u;
+        *alpha_out = alpha;
+    } else {
+        return DQ_ERR_INVALID_ARG;
+    }
+    return DQ_OK;
+}
+
+// cuTensorMapEncodeTiled, looked up at run time so the library loads on machines without a driver.
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_tiled()
+{
+    static encode_tiled_fn fn = []() -> encode_tiled_fn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<encode_tiled_fn>(p);
+    }();
+    return fn;
+}
+
+// [rows x 32 fp32] view of a flat vector, boxes of `box_rows` rows, 128-byte swizzle.
+bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t box_rows)
+{
+    encode_tiled_fn fn = get_encode_tiled();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {32u, rows};
+    const cuuint64_t strides[1] = {128u};
+    const cuuint32_t box[2] = {32u, box_rows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2u, const_cast<float*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int MODE>
+struct EncLaunch {
+    template <int BITS>
+    static cudaError_t tiles(const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid, uint32_t block,
+                             size_t smem, cudaStream_t st)
+    {
+        auto k = dq::encode_tiles_kernel<BITS, MODE>;
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k<<<grid, block, smem, st>>>(map, a);
+        return cudaGetLastError();
+    }
+    template <int BITS>
+    static cudaError_t buckets(const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
+    {
+        dq::encode_buckets_kernel<BITS, MODE><<<grid, 128, 0, st>>>(a);
+        return cudaGetLastError();
+    }
+};
+
+#define DQ_DISPATCH_BITS(bits, CALL)                                                                            \
+    switch (bits) {                                                                                             \
+        case 1: e = CALL(1); break;                                                                             \
+        case 2: e = CALL(2); break;                                                                             \
+        case 3: e = CALL(3); break;                                                                             \
+        case 4: e = CALL(4); break;                                                                             \
+        case 5: e = CALL(5); break;                                                                             \
+        case 6: e = CALL(6); break;                                                                             \
+        case 7: e = CALL(7); break;                                                                             \
+        default: e = CALL(8); break;                                                                            \
+    }
+
+template <int MODE>
+cudaError_t launch_tiles(uint32_t bits, const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid,
+                         uint32_t block, size_t smem, cudaStream_t st)
+{
+    cudaError_t e;
+#define CALL(B) EncLaunch<MODE>::template tiles<B>(map, a, grid, block, smem, st)
+    DQ_DISPATCH_BITS(bits, CALL)
+#undef CALL
+    return e;
+}
+
+template <int MODE>
+cudaError_t launch_buckets(uint32_t bits, const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
+{
+    cudaError_t e;
+#define CALL(B) EncLaunch<MODE>::template buckets<B>(a, grid, st)
+    DQ_DISPATCH_BITS(bits, CALL)
+#undef CALL
+    return e;
+}
+
+dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t seed, uint32_t worker,
+                        uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
+                        cudaStream_t st)
+{
+    uint32_t L = 0;
+    float alpha = 1.0f;
+    dq_status s = check_params(p, kind, &L, &alpha);
+    if (s != DQ_OK) return s;
+    if (n == 0) return DQ_OK;
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    if (!grad || !out_packed || !out_scale) return DQ_ERR_INVALID_ARG;
+    if (!aligned16(grad) || !aligned16(out_packed) || !aligned16(out_scale)) return DQ_ERR_ALIGNMENT;
+
+    dq::EncodeArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.grad = grad;
+    a.packed = out_packed;
+    a.scale = out_scale;
+    a.n = n;
+    a.bucket = p->bucket;
+    a.num_buckets = dq_num_buckets(n, p->bucket);
+    a.num_words = dq_packed_words(n, p->bits);
+    int mode;
+    if (kind == DQ_KIND_DQSG) {
+        mode = dq::kEncDqsg;
+        a.shift = (float)(L - 1u) / 2.0f;
+        a.gain_num = a.shift;
+        a.kmax = (float)(L - 1u);
+    } else {
+        mode = is_pow2(p->coarse_K) ? dq::kEncNdqsgPow2 : dq::kEncNdqsgAnyK;
+        a.gain_num = alpha * p->fine_M;
+        a.K = p->coarse_K;
+        a.K_offset = ((4194304u + p->coarse_K - 1u) / p->coarse_K) * p->coarse_K;
+    }
+    fill_philox(a.ps, seed, worker, step);
+
+    // power-of-two buckets up to 8192: whole tiles of max(B, 1024) elements go through the tile kernel
+    uint64_t done_buckets = 0;
+    const uint32_t B = p->bucket;
+    if (is_pow2(B) && B <= 8192u) {
+        const uint32_t T = (B < 1024u) ? 1024u : B;
+        const uint64_t tiles = n / T;
+        if (tiles > 0) {
+            if (tiles > 0xFFFFFFFFull) return DQ_ERR_UNSUPPORTED;
+            CUtensorMap map;
+            if (!make_row_map(&map, grad, tiles * (T / 32u), T / 32u)) return DQ_ERR_CUDA;
+            a.num_tiles = (uint32_t)tiles;
+            a.rows_per_tile = T / 32u;
+            a.lanes_per_bucket = (B < 1024u) ? (B / 32u) : 32u;
+            uint32_t warps = (T <= 1024u) ? 8u : (T <= 4096u ? 4u : 2u);
+            const size_t smem = (size_t)warps * T * 4u + 1024u;
+            const uint32_t grid = (uint32_t)((tiles + warps - 1u) / warps);
+            cudaError_t e;
+            if (mode == dq::kEncDqsg) e = launch_tiles<dq::kEncDqsg>(p->bits, map, a, grid, warps * 32u, smem, st);
+            else if (mode == dq::kEncNdqsgPow2) e = launch_tiles<dq::kEncNdqsgPow2>(p->bits, map, a, grid, warps * 32u, smem, st);
+            else e = launch_tiles<dq::kEncNdqsgAnyK>(p->bits, map, a, grid, warps * 32u, smem, st);
+            if (e != cudaSuccess) return DQ_ERR_CUDA;
+            g_launches.fetch_add(1);
+            done_buckets = tiles * (T / B);
+        }
+    }
+    if (done_buckets < a.num_buckets) {
+        a.first_bucket = done_buckets;
+        const uint64_t rest = a.num_buckets - done_buckets;
+        const uint64_t grid64 = (rest + 3u) / 4u;
+        if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
+        cudaError_t e;
+        if (mode == dq::kEncDqsg) e = launch_buckets<dq::kEncDqsg>(p->bits, a, (uint32_t)grid64, st);
+        else if (mode == dq::kEncNdqsgPow2) e = launch_buckets<dq::kEncNdqsgPow2>(p->bits, a, (uint32_t)grid64, st);
+        else e = launch_buckets<dq::kEncNdqsgAnyK>(p->bits, a, (uint32_t)grid64, st);
+        if (e != cudaSuccess) return DQ_ERR_CUDA;
+        g_launches.fetch_add(1);
+    }
+    return DQ_OK;
+}
+
+dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, const float* side_info,
+                        float* out_avg, uint32_t* status_word, bool allow_nested, cudaStream_t st)
+{
+    if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
+    static thread_local dq::DecodeArgs a;    // ~10 KB: keep it off the stack
+    std::memset(&a, 0, sizeof(a));
+    bool any_nested = false;
+    for (uint32_t w = 0; w < W; ++w) {
+        const dq_msg& m = msgs[w];
+        uint32_t L = 0;
+        float alpha = 1.0f;
+        dq_status s = check_params(&m.p, m.kind, &L, &alpha);
+        if (s != DQ_OK) return s;
+        if (m.kind == DQ_KIND_NDQSG && !allow_nested) return DQ_ERR_INVALID_ARG;
+        if (m.p.bucket != msgs[0].p.bucket) return DQ_ERR_UNSUPPORTED;
+        dq::DecWorker& d = a.w[w];
+        d.packed = m.packed;
+        d.scale = m.scale;
+        fill_philox(d.ps, m.seed, m.worker, step);
+        d.bits = m.p.bits;
+        if (m.kind == DQ_KIND_DQSG) {
+            d.kind = 0u;
+            d.s = (float)(L - 1u) / 2.0f;
+            d.cconst = 4194304.0f + d.s - 1.5f;
+        } else {
+            any_nested = true;
+            d.kind = 1u;
+            d.K = m.p.coarse_K;
+            d.K_is_pow2 = is_pow2(m.p.coarse_K) ? 1u : 0u;
+            d.cconst = 4194304.0f - 1.5f;
+            d.A = alpha * m.p.fine_M;
+            d.M1 = m.p.fine_M;
+            d.alpha = alpha;
+            const float a2 = alpha * alpha;
+            d.one_m_alpha2 = 1.0f - a2;
+            d.Kf = (float)m.p.coarse_K;
+            d.invK = 1.0f / d.Kf;
+        }
+    }
+    if (n == 0) return DQ_OK;
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    if (!out_avg) return DQ_ERR_INVALID_ARG;
+    if (any_nested && !side_info) return DQ_ERR_INVALID_ARG;
+    if (!aligned16(out_avg) || (side_info && !aligned16(side_info))) return DQ_ERR_ALIGNMENT;
+    for (uint32_t w = 0; w < W; ++w) {
+        if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
+        if (!aligned16(msgs[w].packed) || !aligned16(msgs[w].scale)) return DQ_ERR_ALIGNMENT;
+    }
+    a.side = any_nested ? side_info : nullptr;
+    a.out = out_avg;
+    a.status = status_word;
+    a.n = n;
+    a.rows = (n + 31u) / 32u;
+    a.W = W;
+    a.rows_per_bucket = msgs[0].p.bucket / 32u;
+    a.Wf = (float)W;
+    a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
+    const uint64_t grid64 = (a.rows + 127u) / 128u;
+    if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
+    if (any_nested) dq::decode_aggregate_kernel<true><<<(uint32_t)grid64, 128, 0, st>>>(a);
+    else dq::decode_aggregate_kernel<false><<<(uint32_t)grid64, 128, 0, st>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return DQ_OK;
+}
+
+uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1u) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+uint64_t dq_packed_words(uint64_t n, uint32_t bits) { return (n * (uint64_t)bits + 31u) / 32u; }
+uint64_t dq_num_buckets(uint64_t n, uint32_t bucket) { return bucket ? (n + bucket - 1u) / bucket : 0u; }
+uint32_t dq_default_levels(uint32_t bits) { return bits == 1u ? 2u : (1u << bits) - 1u; }
+
+const char* dq_status_string(dq_status s)
+{
+    switch (s) {
+        case DQ_OK: return "ok";
+        case DQ_ERR_INVALID_ARG: return "invalid argument";
+        case DQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case DQ_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+        case DQ_ERR_CUDA: return "CUDA call failed";
+    }
+    return "unknown status";
+}
+
+dq_status dqsg_encode(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                      const dq_params* p, uint32_t* out_packed, float* out_scale, void* cuda_stream)
+{
+    return encode_common(DQ_KIND_DQSG, grad, n, seed, worker, step, p, out_packed, out_scale,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+dq_status ndqsg_encode(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                       const dq_params* p, uint32_t* out_packed, float* out_scale, void* cuda_stream)
+{
+    return encode_common(DQ_KIND_NDQSG, grad, n, seed, worker, step, p, out_packed, out_scale,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+dq_status dqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, float* out_avg,
+                                void* cuda_stream)
+{
+    return decode_common(msgs, W, n, step, nullptr, out_avg, nullptr, false, static_cast<cudaStream_t>(cuda_stream));
+}
+
+dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                 const float* side_info, float* out_avg, uint32_t* status_word, void* cuda_stream)
+{
+    return decode_common(msgs, W, n, step, side_info, out_avg, status_word, true,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ------------------------------------------------------------------------------------------------ host buffers
+uint64_t dq_encode_workspace_bytes(uint64_t n, const dq_params* p)
+{
+    if (!p || p->bucket == 0u) return 0u;
+    return align_up(n * 4u, 256u) + align_up(dq_packed_words(n, p->bits) * 4u, 256u) +
+           align_up(dq_num_buckets(n, p->bucket) * 4u, 256u);
+}
+
+uint64_t dq_decode_workspace_bytes(const dq_msg* msgs, uint32_t W, uint64_t n, int has_side_info)
+{
+    if (!msgs) return 0u;
+    uint64_t total = align_up(n * 4u, 256u) * (has_side_info ? 2u : 1u);
+    for (uint32_t w = 0; w < W; ++w) {
+        if (msgs[w].p.bucket == 0u) return 0u;
+        total += align_up(dq_packed_words(n, msgs[w].p.bits) * 4u, 256u) +
+                 align_up(dq_num_buckets(n, msgs[w].p.bucket) * 4u, 256u);
+    }
+    return total;
+}
+
+static dq_status encode_host(dq_kind kind, const float* grad, uint64_t n, uint64_t seed, uint32_t worker,
+                             uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
+                             void* workspace, uint64_t workspace_bytes, void* cuda_stream)
+{
+    uint32_t L;
+    float alpha;
+    dq_status s = check_params(p, kind, &L, &alpha);
+    if (s != DQ_OK) return s;
+    if (n == 0) return DQ_OK;
+    if (!grad || !out_packed || !out_scale || !workspace) return DQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0u) return DQ_ERR_ALIGNMENT;
+    if (workspace_bytes < dq_encode_workspace_bytes(n, p)) return DQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    float* d_grad = reinterpret_cast<float*>(ws);
+    ws += align_up(n * 4u, 256u);
+    uint32_t* d_packed = reinterpret_cast<uint32_t*>(ws);
+    const uint64_t pbytes = dq_packed_words(n, p->bits) * 4u;
+    ws += align_up(pbytes, 256u);
+    float* d_scale = reinterpret_cast<float*>(ws);
+    const uint64_t sbytes = dq_num_buckets(n, p->bucket) * 4u;
+    if (cudaMemcpyAsync(d_grad, grad, n * 4u, cudaMemcpyHostToDevice, st) != cudaSuccess) return DQ_ERR_CUDA;
+    s = encode_common(kind, d_grad, n, seed, worker, step, p, d_packed, d_scale, st);
+    if (s != DQ_OK) return s;
+    if (cudaMemcpyAsync(out_packed, d_packed, pbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpyAsync(out_scale, d_scale, sbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+dq_status dqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                           const dq_params* p, uint32_t* out_packed, float* out_scale, void* workspace,
+                           uint64_t workspace_bytes, void* cuda_stream)
+{
+    return encode_host(DQ_KIND_DQSG, grad, n, seed, worker, step, p, out_packed, out_scale, workspace,
+                       workspace_bytes, cuda_stream);
+}
+
+dq_status ndqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                            const dq_params* p, uint32_t* out_packed, float* out_scale, void* workspace,
+                            uint64_t workspace_bytes, void* cuda_stream)
+{
+    return encode_host(DQ_KIND_NDQSG, grad, n, seed, worker, step, p, out_packed, out_scale, workspace,
+                       workspace_bytes, cuda_stream);
+}
+
+dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                      const float* side_info, float* out_avg, void* workspace,
+                                      uint64_t workspace_bytes, void* cuda_stream)
+{
+    if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
+    for (uint32_t w = 0; w < W; ++w) {
+        uint32_t L;
+        float alpha;
+        dq_status s = check_params(&msgs[w].p, msgs[w].kind, &L, &alpha);
+        if (s != DQ_OK) return s;
+        if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
+    }
+    if (n == 0) return DQ_OK;
+    if (!out_avg || !workspace) return DQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0u) return DQ_ERR_ALIGNMENT;
+    if (workspace_bytes < dq_decode_workspace_bytes(msgs, W, n, side_info != nullptr)) return DQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    float* d_out = reinterpret_cast<float*>(ws);
+    ws += align_up(n * 4u, 256u);
+    float* d_side = nullptr;
+    if (side_info) {
+        d_side = reinterpret_cast<float*>(ws);
+        ws += align_up(n * 4u, 256u);
+        if (cudaMemcpyAsync(d_side, side_info, n * 4u, cudaMemcpyHostToDevice, st) != cudaSuccess) return DQ_ERR_CUDA;
+    }
+    dq_msg dev_msgs[DQ_MAX_WORKERS];
+    for (uint32_t w = 0; w < W; ++w) {
+        dev_msgs[w] = msgs[w];
+        const uint64_t pbytes = dq_packed_words(n, msgs[w].p.bits) * 4u;
+        const uint64_t sbytes = dq_num_buckets(n, msgs[w].p.bucket) * 4u;
+        uint32_t* d_p = reinterpret_cast<uint32_t*>(ws);
+        ws += align_up(pbytes, 256u);
+        float* d_s = reinterpret_cast<float*>(ws);
+        ws += align_up(sbytes, 256u);
+        if (cudaMemcpyAsync(d_p, msgs[w].packed, pbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return DQ_ERR_CUDA;
+        if (cudaMemcpyAsync(d_s, msgs[w].scale, sbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return DQ_ERR_CUDA;
+        dev_msgs[w].packed = d_p;
+        dev_msgs[w].scale = d_s;
+    }
+    dq_status s = decode_common(dev_msgs, W, n, step, d_side, d_out, nullptr, true, st);
+    if (s != DQ_OK) return s;
+    if (cudaMemcpyAsync(out_avg, d_out, n * 4u, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+dq_status dq_device_error_flags(uint32_t* out_flags)
+{
+    if (!out_flags) return DQ_ERR_INVALID_ARG;
+    unsigned int v = 0u, zero = 0u;
+    if (cudaDeviceSynchronize() != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, dq::g_dq_error_flags, sizeof(v)) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpyToSymbol(dq::g_dq_error_flags, &zero, sizeof(zero)) != cudaSuccess) return DQ_ERR_CUDA;
+    *out_flags = v;
+    return DQ_OK;
+}
+
+uint64_t dq_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

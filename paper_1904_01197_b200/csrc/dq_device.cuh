@@ -1,0 +1,111 @@
+// Device-side building blocks shared by the encode and decode kernels: the Philox4x32-10 dither stream,
+// the bit-pattern tricks that replace int<->float conversions, and the asynchronous tile copy (TMA)
+// wrappers.  sm_100a only.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dq {
+
+// ---------------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  The ten round keys (key + r * Weyl constant) are computed on the
+// host and travel as kernel parameters, so the logic ops read them straight from the constant bank.
+// ---------------------------------------------------------------------------------------------------
+constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
+constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
+constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
+
+struct PhiloxStream {
+    uint32_t rk[10][2];   // round keys
+    uint32_t c1, c2, c3;  // counter words 1..3: worker, lo32(step), hi32(step)
+};
+
+// One block: counter word 0 is the index of the 4-element chunk (element index / 4).
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, const PhiloxStream& ps, uint32_t (&out)[4])
+{
+    uint32_t c1 = ps.c1, c2 = ps.c2, c3 = ps.c3;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0;
+        const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ ps.rk[r][0];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ ps.rk[r][1];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// 32 random bits -> f in [1, 2) on the odd grid; the dither in fine-step units is f - 1.5 (exact).
+__device__ __forceinline__ float dither_f12(uint32_t x)
+{
+    return __uint_as_float((x >> 9) | 0x3F800001u);
+}
+
+// Round-to-nearest-even of |w| < 2^22 by adding 1.5 * 2^23: the integer lands in the low mantissa bits.
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
+constexpr uint32_t kMagicBits = 0x4B400000u;   // bit pattern of kMagic
+
+// ---------------------------------------------------------------------------------------------------
+// Asynchronous tile copies (TMA) with an mbarrier, and a bounded wait.
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void fence_mbar_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// Load a [rows x 32 floats] box whose first row is `row0` into shared memory (128-byte swizzle).
+__device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap* tmap, uint32_t bar, int32_t row0)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"((uint64_t)tmap), "r"(bar), "r"(0), "r"(row0)
+        : "memory");
+}
+
+// Waits for phase `parity` of the barrier; gives up after a fixed number of tries (each try itself blocks
+// for a hardware-defined time), so a copy that never lands cannot hang the kernel.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+
+// Byte offset, inside a 128-byte-swizzled tile of 128-byte rows, of 16-byte chunk `c` of row `r`.
+__device__ __forceinline__ uint32_t swz128(uint32_t r, uint32_t c)
+{
+    return r * 128u + ((c ^ (r & 7u)) << 4);
+}
+
+}  // namespace dq
