@@ -27,6 +27,29 @@ void fill_philox(dq::PhiloxStream& ps, uint64_t seed, uint32_t worker, uint64_t 
     ps.c1 = worker;
     ps.c2 = (uint32_t)(step & 0xFFFFFFFFull);
     ps.c3 = (uint32_t)(step >> 32);
+    // the block-independent parts of rounds 0..2 (see PhiloxStream)
+    const uint64_t p1 = (uint64_t)dq::kPhiloxM1 * (uint64_t)ps.c2;
+    const uint32_t u0 = (uint32_t)(p1 >> 32) ^ ps.c1 ^ ps.rk[0][0];
+    const uint32_t u1 = (uint32_t)p1;
+    const uint64_t p0 = (uint64_t)dq::kPhiloxM0 * (uint64_t)u0;
+    ps.v0 = ps.c3 ^ ps.rk[0][1];
+    ps.v1 = u1 ^ ps.rk[1][0];
+    ps.v2 = (uint32_t)(p0 >> 32) ^ ps.rk[1][1];
+    ps.v3 = (uint32_t)p0 ^ ps.rk[2][1];
+}
+
+int device_sm_count()
+{
+    static thread_local int cached_dev = -1, cached_sms = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (dev != cached_dev) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached_dev = dev;
+        cached_sms = sms;
+    }
+    return cached_sms;
 }
 
 dq_status check_params(const dq_params* p, dq_kind kind, uint32_t* levels_out, float* alpha_out)
@@ -86,57 +109,34 @@ bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int MODE>
-struct EncLaunch {
-    template <int BITS>
-    static cudaError_t tiles(const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid, uint32_t block,
-                             size_t smem, cudaStream_t st)
-    {
-        auto k = dq::encode_tiles_kernel<BITS, MODE>;
-        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        k<<<grid, block, smem, st>>>(map, a);
-        return cudaGetLastError();
-    }
-    template <int BITS>
-    static cudaError_t buckets(const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
-    {
-        dq::encode_buckets_kernel<BITS, MODE><<<grid, 128, 0, st>>>(a);
-        return cudaGetLastError();
-    }
-};
-
-#define DQ_DISPATCH_BITS(bits, CALL)                                                                            \
-    switch (bits) {                                                                                             \
-        case 1: e = CALL(1); break;                                                                             \
-        case 2: e = CALL(2); break;                                                                             \
-        case 3: e = CALL(3); break;                                                                             \
-        case 4: e = CALL(4); break;                                                                             \
-        case 5: e = CALL(5); break;                                                                             \
-        case 6: e = CALL(6); break;                                                                             \
-        case 7: e = CALL(7); break;                                                                             \
-        default: e = CALL(8); break;                                                                            \
-    }
-
-template <int MODE>
-cudaError_t launch_tiles(uint32_t bits, const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid,
-                         uint32_t block, size_t smem, cudaStream_t st)
+template <int MODE, int BITS>
+cudaError_t launch_encode_one(const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
 {
-    cudaError_t e;
-#define CALL(B) EncLaunch<MODE>::template tiles<B>(map, a, grid, block, smem, st)
-    DQ_DISPATCH_BITS(bits, CALL)
-#undef CALL
-    return e;
+    auto k = dq::encode_kernel<BITS, MODE>;
+    static thread_local bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dq::kEncSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    k<<<grid, dq::kEncThreads, dq::kEncSmemBytes, st>>>(map, a);
+    return cudaGetLastError();
 }
 
 template <int MODE>
-cudaError_t launch_buckets(uint32_t bits, const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
+cudaError_t launch_encode(uint32_t bits, const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid,
+                          cudaStream_t st)
 {
-    cudaError_t e;
-#define CALL(B) EncLaunch<MODE>::template buckets<B>(a, grid, st)
-    DQ_DISPATCH_BITS(bits, CALL)
-#undef CALL
-    return e;
+    switch (bits) {
+        case 1: return launch_encode_one<MODE, 1>(map, a, grid, st);
+        case 2: return launch_encode_one<MODE, 2>(map, a, grid, st);
+        case 3: return launch_encode_one<MODE, 3>(map, a, grid, st);
+        case 4: return launch_encode_one<MODE, 4>(map, a, grid, st);
+        case 5: return launch_encode_one<MODE, 5>(map, a, grid, st);
+        case 6: return launch_encode_one<MODE, 6>(map, a, grid, st);
+        case 7: return launch_encode_one<MODE, 7>(map, a, grid, st);
+        default: return launch_encode_one<MODE, 8>(map, a, grid, st);
+    }
 }
 
 dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t seed, uint32_t worker,
@@ -175,43 +175,47 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     }
     fill_philox(a.ps, seed, worker, step);
 
-    // power-of-two buckets up to 8192: whole tiles of max(B, 1024) elements go through the tile kernel
-    uint64_t done_buckets = 0;
+    // power-of-two buckets up to 8192: whole tiles of 8192 elements go through the tile path of the kernel,
+    // the rest (and every other bucket size) through its plain-load part, in the same launch
+    const int sms = device_sm_count();
+    if (sms <= 0) return DQ_ERR_CUDA;
     const uint32_t B = p->bucket;
-    if (is_pow2(B) && B <= 8192u) {
-        const uint32_t T = (B < 1024u) ? 1024u : B;
-        const uint64_t tiles = n / T;
-        if (tiles > 0) {
-            if (tiles > 0xFFFFFFFFull) return DQ_ERR_UNSUPPORTED;
-            CUtensorMap map;
-            if (!make_row_map(&map, grad, tiles * (T / 32u), T / 32u)) return DQ_ERR_CUDA;
-            a.num_tiles = (uint32_t)tiles;
-            a.rows_per_tile = T / 32u;
-            a.lanes_per_bucket = (B < 1024u) ? (B / 32u) : 32u;
-            uint32_t warps = (T <= 1024u) ? 8u : (T <= 4096u ? 4u : 2u);
-            const size_t smem = (size_t)warps * T * 4u + 1024u;
-            const uint32_t grid = (uint32_t)((tiles + warps - 1u) / warps);
-            cudaError_t e;
-            if (mode == dq::kEncDqsg) e = launch_tiles<dq::kEncDqsg>(p->bits, map, a, grid, warps * 32u, smem, st);
-            else if (mode == dq::kEncNdqsgPow2) e = launch_tiles<dq::kEncNdqsgPow2>(p->bits, map, a, grid, warps * 32u, smem, st);
-            else e = launch_tiles<dq::kEncNdqsgAnyK>(p->bits, map, a, grid, warps * 32u, smem, st);
-            if (e != cudaSuccess) return DQ_ERR_CUDA;
-            g_launches.fetch_add(1);
-            done_buckets = tiles * (T / B);
-        }
+    const uint32_t T = (uint32_t)dq::kTileRows * 32u;
+    uint64_t tiles = (is_pow2(B) && B <= T) ? n / T : 0u;
+    if (tiles > 0xFFFFFFFFull) return DQ_ERR_UNSUPPORTED;
+    CUtensorMap map;
+    std::memset(&map, 0, sizeof(map));
+    if (tiles > 0) {
+        if (!make_row_map(&map, grad, tiles * dq::kTileRows, dq::kTileRows)) return DQ_ERR_CUDA;
+        a.num_tiles = (uint32_t)tiles;
+        a.lanes_per_bucket = (B < 1024u) ? (B / 32u) : 32u;
+        a.warps_per_bucket = (B < 1024u) ? 1u : (B / 1024u);
+        uint32_t lg = 0;
+        while ((1u << lg) < B) ++lg;
+        a.bucket_log2 = lg;
     }
-    if (done_buckets < a.num_buckets) {
-        a.first_bucket = done_buckets;
-        const uint64_t rest = a.num_buckets - done_buckets;
-        const uint64_t grid64 = (rest + 3u) / 4u;
-        if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
-        cudaError_t e;
-        if (mode == dq::kEncDqsg) e = launch_buckets<dq::kEncDqsg>(p->bits, a, (uint32_t)grid64, st);
-        else if (mode == dq::kEncNdqsgPow2) e = launch_buckets<dq::kEncNdqsgPow2>(p->bits, a, (uint32_t)grid64, st);
-        else e = launch_buckets<dq::kEncNdqsgAnyK>(p->bits, a, (uint32_t)grid64, st);
-        if (e != cudaSuccess) return DQ_ERR_CUDA;
-        g_launches.fetch_add(1);
+    a.first_bucket = tiles * (T / B);
+    const uint64_t rest = a.num_buckets - a.first_bucket;
+    const uint32_t slots = 3u * (uint32_t)sms;                      // resident CTAs (3 per SM)
+    uint32_t plain = 0;
+    if (rest > 0) {
+        const uint64_t want = (rest + dq::kConsumerWarps - 1u) / dq::kConsumerWarps;
+        const uint64_t cap = (tiles > 0) ? (slots / 4u) : (4ull * slots);
+        plain = (uint32_t)(want < cap ? want : cap);
+        if (plain == 0u) plain = 1u;
     }
+    a.plain_ctas = plain;
+    uint32_t tile_ctas = 0;
+    if (tiles > 0) {
+        const uint32_t room = (slots > plain) ? (slots - plain) : 1u;
+        tile_ctas = (uint32_t)(tiles < room ? tiles : room);
+    }
+    cudaError_t e;
+    if (mode == dq::kEncDqsg) e = launch_encode<dq::kEncDqsg>(p->bits, map, a, plain + tile_ctas, st);
+    else if (mode == dq::kEncNdqsgPow2) e = launch_encode<dq::kEncNdqsgPow2>(p->bits, map, a, plain + tile_ctas, st);
+    else e = launch_encode<dq::kEncNdqsgAnyK>(p->bits, map, a, plain + tile_ctas, st);
+    if (e != cudaSuccess) return DQ_ERR_CUDA;
+    g_launches.fetch_add(1);
     return DQ_OK;
 }
 
@@ -236,14 +240,13 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         fill_philox(d.ps, m.seed, m.worker, step);
         d.bits = m.p.bits;
         if (m.kind == DQ_KIND_DQSG) {
-            d.kind = 0u;
+            d.kind = dq::kDecDqsg;
             d.s = (float)(L - 1u) / 2.0f;
             d.cconst = 4194304.0f + d.s - 1.5f;
         } else {
             any_nested = true;
-            d.kind = 1u;
-            d.K = m.p.coarse_K;
-            d.K_is_pow2 = is_pow2(m.p.coarse_K) ? 1u : 0u;
+            if (!is_pow2(m.p.coarse_K)) d.kind = dq::kDecNdqsgAnyK;
+            else d.kind = (alpha == 1.0f) ? dq::kDecNdqsgPow2 : dq::kDecNdqsgPow2Shrink;
             d.cconst = 4194304.0f - 1.5f;
             d.A = alpha * m.p.fine_M;
             d.M1 = m.p.fine_M;
@@ -272,10 +275,9 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.rows_per_bucket = msgs[0].p.bucket / 32u;
     a.Wf = (float)W;
     a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
-    const uint64_t grid64 = (a.rows + 127u) / 128u;
+    const uint64_t grid64 = (a.rows + dq::kDecThreads - 1u) / dq::kDecThreads;
     if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
-    if (any_nested) dq::decode_aggregate_kernel<true><<<(uint32_t)grid64, 128, 0, st>>>(a);
-    else dq::decode_aggregate_kernel<false><<<(uint32_t)grid64, 128, 0, st>>>(a);
+    dq::decode_aggregate_kernel<<<(uint32_t)grid64, dq::kDecThreads, 0, st>>>(a);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;

@@ -3,22 +3,27 @@
 //
 // One lane owns one row = 32 consecutive elements: 32 fp32 accumulators in registers, and per worker
 // exactly `bits` packed words.  For every worker (in array order) the lane reloads that worker's words and
-// bucket scale, regenerates the 32 dithers with eight Philox blocks, reconstructs and accumulates; the mean
-// is written at the end.  The packed streams, the side information and the output are each touched once.
+// bucket scale, regenerates the 32 dithers (Philox blocks four at a time, so four dependency chains are in
+// flight), reconstructs and accumulates; the mean is written at the end.  The packed streams, the side
+// information and the output are each touched once in HBM (the side information is re-read per worker from
+// L1, which keeps it out of the register file).
+//
+// The path is bound by instruction issue, not by HBM: each (element, worker) pair needs a quarter of a
+// Philox block (9.25 integer instructions) before any reconstruction arithmetic.
 #pragma once
 
 #include "dq_device.cuh"
 
 namespace dq {
 
+enum DecKind : uint32_t { kDecDqsg = 0, kDecNdqsgPow2 = 1, kDecNdqsgPow2Shrink = 2, kDecNdqsgAnyK = 3 };
+
 struct DecWorker {
     const uint32_t* packed;
     const float* scale;
     PhiloxStream ps;
-    uint32_t kind;        // 0 DQSG, 1 NDQSG
+    uint32_t kind;        // DecKind
     uint32_t bits;
-    uint32_t K;           // NDQSG coarse ratio
-    uint32_t K_is_pow2;
     float s;              // DQSG (L-1)/2
     float cconst;         // DQSG: 4194304 + s - 1.5 ; NDQSG: 4194304 - 1.5   (see unpack_half_biased)
     float A;              // NDQSG alpha * M1
@@ -42,8 +47,9 @@ struct DecodeArgs {
     DecWorker w[64];
 };
 
-// Code of element `idx` of a row, returned as the bit pattern of the float 2^22 + code (code in mantissa
-// bits 1.., since floats in [2^22, 2^23) step by 1/2).  Subtracting a constant then gives code - c exactly.
+// Code of element `idx` of a row, returned as the float 2^22 + code/1 ... precisely: the bit pattern of
+// 2^22 with the code in mantissa bits 1.., i.e. the value 2^22 + code (floats in [2^22, 2^23) step by 1/2).
+// Subtracting a constant then gives code - c exactly.
 template <int BITS>
 __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS], int idx)
 {
@@ -61,13 +67,9 @@ __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS
 }
 
 template <int BITS>
-__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
-                                           uint64_t n, const float (&y)[32], float (&acc)[32],
-                                           uint32_t* status)
+__device__ __forceinline__ void load_row_words(const uint32_t* src, bool full_row, uint64_t first_word,
+                                               uint64_t num_words, uint32_t (&words)[BITS])
 {
-    // this worker's words for the row
-    uint32_t words[BITS];
-    const uint32_t* src = wk.packed + row * BITS;
     if (full_row) {
         if constexpr (BITS % 4 == 0) {
 #pragma unroll
@@ -86,60 +88,105 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
             for (int j = 0; j < BITS; ++j) words[j] = __ldg(src + j);
         }
     } else {
-        const uint64_t num_words = (n * BITS + 31u) >> 5;
 #pragma unroll
-        for (int j = 0; j < BITS; ++j) words[j] = (row * BITS + j < num_words) ? __ldg(src + j) : 0u;
+        for (int j = 0; j < BITS; ++j) words[j] = (first_word + j < num_words) ? __ldg(src + j) : 0u;
     }
+}
+
+// One worker's contribution to the 32 accumulators of a row.
+//   DQSG:  g~ = (kappa/s) ((k - s) - delta); (k - s + 1.5) - f rounds once to the same value.
+//   NDQSG: r = (m - delta) - y a;  jj = rint(r / K);  q1^ = m - K jj;  g~ = beta (q1^ - delta) [+ (1-alpha^2) y]
+template <int BITS, uint32_t KIND>
+__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
+                                           uint64_t n, const float* __restrict__ side_row, float (&acc)[32],
+                                           uint32_t* status)
+{
+    uint32_t words[BITS];
+    load_row_words<BITS>(wk.packed + row * BITS, full_row, row * BITS, (n * BITS + 31u) >> 5, words);
 
     const float kappa = __ldg(wk.scale + bucket);
     if (status != nullptr && !(fabsf(kappa) <= 3.402823466e38f)) atomicOr(status, 0x1u);
 
-    const uint32_t chunk0 = (uint32_t)(row * 8u);
-    if (wk.kind == 0u) {
-        // g~ = (kappa/s) ((k - s) - delta), with (k - s + 1.5) - f == (k - s) - delta after one rounding
-        const float c = __fdiv_rn(kappa, wk.s);
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            uint32_t rnd[4];
-            philox4x32_10(chunk0 + (uint32_t)ch, wk.ps, rnd);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int idx = 4 * ch + e;
-                const float X = __fadd_rn(unpack_half_biased<BITS>(words, idx), -wk.cconst);   // k - s + 1.5
-                const float d = __fadd_rn(X, -dither_f12(rnd[e]));
-                acc[idx] = __fadd_rn(acc[idx], __fmul_rn(c, d));
-            }
-        }
+    float c, a = 0.0f;
+    if (KIND == kDecDqsg) {
+        c = __fdiv_rn(kappa, wk.s);
     } else {
-        const float a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
-        const float beta = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);
-        const bool shrink = (wk.alpha != 1.0f);
+        a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
+        c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);                 // beta
+    }
+    const uint32_t chunk0 = (uint32_t)(row * 8u);
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            uint32_t rnd[4];
-            philox4x32_10(chunk0 + (uint32_t)ch, wk.ps, rnd);
+    for (int h = 0; h < 2; ++h) {
+        uint32_t ctr[4], rnd[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ctr[j] = chunk0 + (uint32_t)(4 * h + j);
+        philox4x32_10_xN<4>(ctr, wk.ps, rnd);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            if (KIND != kDecDqsg) {
+                if (full_row) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + 4 * h + j);
+                    y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        y[e] = (row * 32u + 16u * h + 4u * j + e < n) ? __ldg(side_row + 16 * h + 4 * j + e) : 0.0f;
+                }
+            }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int idx = 4 * ch + e;
-                const float f = dither_f12(rnd[e]);
-                const float X1 = __fadd_rn(unpack_half_biased<BITS>(words, idx), -wk.cconst);  // m + 1.5
-                const float r1 = __fadd_rn(X1, -f);                                            // m - delta
-                const float r = __fmaf_rn(-y[idx], a, r1);
-                const float t = wk.K_is_pow2 ? __fmul_rn(r, wk.invK) : __fdiv_rn(r, wk.Kf);
-                const float jj = __fadd_rn(__fadd_rn(t, kMagic), -kMagic);                     // rint(r / K)
-                const float Y = __fmaf_rn(-wk.Kf, jj, X1);                                     // q1^ + 1.5, exact
-                const float d = __fadd_rn(Y, -f);                                              // q1^ - delta
+                const int idx = 16 * h + 4 * j + e;
+                const float f = dither_f12(rnd[j][e]);
+                const float X = __fadd_rn(unpack_half_biased<BITS>(words, idx), -wk.cconst);
                 float gt;
-                if (shrink) gt = __fmaf_rn(beta, d, __fmul_rn(wk.one_m_alpha2, y[idx]));
-                else gt = __fmul_rn(beta, d);
+                if (KIND == kDecDqsg) {
+                    const float d = __fadd_rn(X, -f);                      // (k - s) - delta
+                    gt = __fmul_rn(c, d);
+                } else {
+                    const float yy = y[e];
+                    const float r1 = __fadd_rn(X, -f);                     // m - delta
+                    const float r = __fmaf_rn(-yy, a, r1);
+                    float jj;
+                    if (KIND == kDecNdqsgAnyK) {
+                        jj = __fadd_rn(__fadd_rn(__fdiv_rn(r, wk.Kf), kMagic), -kMagic);
+                    } else {
+                        // K is a power of two: r * (1/K) is exact, so one rounding gives rint(r / K)
+                        jj = __fadd_rn(__fmaf_rn(r, wk.invK, kMagic), -kMagic);
+                    }
+                    const float Y = __fmaf_rn(-wk.Kf, jj, X);              // q1^ + 1.5, exact
+                    const float d = __fadd_rn(Y, -f);                      // q1^ - delta
+                    if (KIND == kDecNdqsgPow2) gt = __fmul_rn(c, d);                          // alpha == 1
+                    else if (KIND == kDecNdqsgPow2Shrink) gt = __fmaf_rn(c, d, __fmul_rn(wk.one_m_alpha2, yy));
+                    else if (wk.alpha == 1.0f) gt = __fmul_rn(c, d);
+                    else gt = __fmaf_rn(c, d, __fmul_rn(wk.one_m_alpha2, yy));
+                }
                 acc[idx] = __fadd_rn(acc[idx], gt);
             }
         }
     }
 }
 
-template <bool HAS_SIDE>
-__global__ void __launch_bounds__(128)
+template <uint32_t KIND>
+__device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
+                                                uint64_t n, const float* side_row, float (&acc)[32],
+                                                uint32_t* status)
+{
+    switch (wk.bits) {
+        case 1: decode_row<1, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 2: decode_row<2, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 3: decode_row<3, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 4: decode_row<4, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 5: decode_row<5, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 6: decode_row<6, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 7: decode_row<7, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        default: decode_row<8, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+    }
+}
+
+constexpr int kDecThreads = 128;
+
+__global__ void __launch_bounds__(kDecThreads, 4)
 decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
 {
     const uint64_t row = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -148,35 +195,19 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     const bool full_row = (base + 32u <= args.n);
     const uint32_t nvalid = full_row ? 32u : (uint32_t)(args.n - base);
     const uint64_t bucket = row / args.rows_per_bucket;
+    const float* side_row = args.side ? args.side + base : nullptr;
 
-    float y[32];
     float acc[32];
 #pragma unroll
-    for (int e = 0; e < 32; ++e) { acc[e] = 0.0f; y[e] = 0.0f; }
-    if (HAS_SIDE) {
-        if (full_row) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(args.side + base) + c);
-                y[4 * c] = v.x; y[4 * c + 1] = v.y; y[4 * c + 2] = v.z; y[4 * c + 3] = v.w;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) y[e] = ((uint32_t)e < nvalid) ? __ldg(args.side + base + e) : 0.0f;
-        }
-    }
+    for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
 
     for (uint32_t w = 0; w < args.W; ++w) {
         const DecWorker& wk = args.w[w];
-        switch (wk.bits) {
-            case 1: decode_row<1>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            case 2: decode_row<2>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            case 3: decode_row<3>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            case 4: decode_row<4>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            case 5: decode_row<5>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            case 6: decode_row<6>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            case 7: decode_row<7>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
-            default: decode_row<8>(wk, row, bucket, full_row, args.n, y, acc, args.status); break;
+        switch (wk.kind) {
+            case kDecDqsg: decode_row_bits<kDecDqsg>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            default: decode_row_bits<kDecNdqsgAnyK>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
         }
     }
 

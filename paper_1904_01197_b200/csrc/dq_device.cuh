@@ -21,24 +21,69 @@ constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 struct PhiloxStream {
     uint32_t rk[10][2];   // round keys
     uint32_t c1, c2, c3;  // counter words 1..3: worker, lo32(step), hi32(step)
+    // Only counter word 0 differs between blocks, so parts of rounds 0..2 are the same for every block of a
+    // (seed, worker, step) stream; the host folds them into four words:
+    uint32_t v0;          // c3 ^ rk[0][1]
+    uint32_t v1;          // lo(M1*c2) ^ rk[1][0]
+    uint32_t v2;          // hi(M0*u0) ^ rk[1][1],  u0 = hi(M1*c2) ^ c1 ^ rk[0][0]
+    uint32_t v3;          // lo(M0*u0) ^ rk[2][1]
 };
 
-// One block: counter word 0 is the index of the 4-element chunk (element index / 4).
+// N blocks at once, rounds outermost, so N independent dependency chains are in flight.
+// Counter word 0 of block j is c0[j] = index of its 4-element chunk (element index / 4).
+template <int N>
+__device__ __forceinline__ void philox4x32_10_xN(const uint32_t (&c0in)[N], const PhiloxStream& ps,
+                                                 uint32_t (&out)[N][4])
+{
+    uint32_t c0[N], c1[N], c2[N], c3[N];
+    // round 0: only M0*c0 depends on the block
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0in[j];
+        c2[j] = (uint32_t)(p0 >> 32) ^ ps.v0;
+        c3[j] = (uint32_t)p0;
+    }
+    // round 1: c0, c1 are still block-independent
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2[j];
+        c0[j] = (uint32_t)(p1 >> 32) ^ ps.v1;
+        c1[j] = (uint32_t)p1;
+        c2[j] = c3[j] ^ ps.v2;
+    }
+    // round 2: c3 is block-independent (folded into v3)
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0[j];
+        const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2[j];
+        c0[j] = (uint32_t)(p1 >> 32) ^ c1[j] ^ ps.rk[2][0];
+        c1[j] = (uint32_t)p1;
+        c2[j] = (uint32_t)(p0 >> 32) ^ ps.v3;
+        c3[j] = (uint32_t)p0;
+    }
+#pragma unroll
+    for (int r = 3; r < 10; ++r) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0[j];
+            const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2[j];
+            c0[j] = (uint32_t)(p1 >> 32) ^ c1[j] ^ ps.rk[r][0];
+            c1[j] = (uint32_t)p1;
+            c2[j] = (uint32_t)(p0 >> 32) ^ c3[j] ^ ps.rk[r][1];
+            c3[j] = (uint32_t)p0;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < N; ++j) { out[j][0] = c0[j]; out[j][1] = c1[j]; out[j][2] = c2[j]; out[j][3] = c3[j]; }
+}
+
+// One block (reference form, all ten rounds written out).
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, const PhiloxStream& ps, uint32_t (&out)[4])
 {
-    uint32_t c1 = ps.c1, c2 = ps.c2, c3 = ps.c3;
-#pragma unroll
-    for (int r = 0; r < 10; ++r) {
-        const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0;
-        const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2;
-        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ ps.rk[r][0];
-        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ ps.rk[r][1];
-        c1 = (uint32_t)p1;
-        c3 = (uint32_t)p0;
-        c0 = n0;
-        c2 = n2;
-    }
-    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+    const uint32_t in[1] = {c0};
+    uint32_t o[1][4];
+    philox4x32_10_xN<1>(in, ps, o);
+    out[0] = o[0][0]; out[1] = o[0][1]; out[2] = o[0][2]; out[3] = o[0][3];
 }
 
 // 32 random bits -> f in [1, 2) on the odd grid; the dither in fine-step units is f - 1.5 (exact).
@@ -86,9 +131,9 @@ __device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap* t
 
 // Waits for phase `parity` of the barrier; gives up after a fixed number of tries (each try itself blocks
 // for a hardware-defined time), so a copy that never lands cannot hang the kernel.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_tries = (1u << 22))
 {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
+    for (uint32_t it = 0; it < max_tries; ++it) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -100,6 +145,17 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         if (ok) return true;
     }
     return false;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Named barrier over `threads` threads (a multiple of 32); id 1..15 (0 is __syncthreads).
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // Byte offset, inside a 128-byte-swizzled tile of 128-byte rows, of 16-byte chunk `c` of row `r`.

@@ -1,15 +1,19 @@
-// Encode kernels: per-bucket scale, dither, quantize, (coset), pack -- all in one pass over the gradient
+// Encode kernel: per-bucket scale, dither, quantize, (coset), pack -- one pass over the gradient
 // (Eq. (DQSG) and Algorithm 1, worker steps; nested encoder equation and Algorithm 2, workers in P2).
 //
 // Work decomposition: a "row" is 32 consecutive elements = one 128-byte line of the gradient and exactly
-// `bits` 32-bit words of the bit stream.  One lane quantizes and packs whole rows, so no lane ever shares a
-// packed word with another lane.
-//   * encode_tiles_kernel: power-of-two buckets.  A warp owns a tile of max(B, 1024) elements; the tile is
-//     brought into shared memory by one asynchronous 2-D tile copy with the 128-byte swizzle, which makes
-//     "lane r reads row r" free of bank conflicts.  Pass 1 reduces max|g| per bucket with warp shuffles,
-//     pass 2 re-reads the tile from shared memory, so the gradient is read from HBM exactly once.
-//   * encode_buckets_kernel: any bucket size, the ragged tail, and everything the tile kernel leaves over;
-//     plain loads, one warp per bucket.
+// `bits` 32-bit words of the bit stream.  One lane quantizes and packs a whole row, so no lane ever shares a
+// packed word with another lane and no shuffles are needed for packing.
+//
+// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight consumer warps plus one
+// producer warp walk over tiles of 8192 elements (256 rows).  The producer keeps a ring of shared-memory
+// stages filled with asynchronous 2-D tile copies (128-byte swizzle, which makes "lane r reads row r" free of
+// bank conflicts).  A consumer warp takes its 32 rows of a stage into registers, hands the stage back at
+// once, reduces max|g| over its bucket (shuffles inside the warp, a named barrier between the warps that
+// share a bucket) and then quantizes from registers.  The gradient is read from HBM exactly once.
+//
+// Everything else -- other bucket sizes, the part of the vector past the last whole tile, the ragged end --
+// is handled by plain-load code, one warp per bucket, in extra CTAs of the same launch.
 #pragma once
 
 #include "dq_device.cuh"
@@ -18,20 +22,29 @@ namespace dq {
 
 enum EncMode : int { kEncDqsg = 0, kEncNdqsgPow2 = 1, kEncNdqsgAnyK = 2 };
 
+constexpr int kTileRows = 256;                     // rows per tile (8192 elements, 32 KB)
+constexpr int kTileBytes = kTileRows * 128;
+constexpr int kConsumerWarps = kTileRows / 32;     // one row per lane
+constexpr int kEncThreads = 32 * (kConsumerWarps + 1);
+constexpr int kEncStages = 2;
+constexpr size_t kEncSmemBytes = (size_t)kEncStages * kTileBytes + 1024;
+
 struct EncodeArgs {
-    const float* grad;       // only used by encode_buckets_kernel
+    const float* grad;
     uint32_t* packed;
     float* scale;
     uint64_t n;              // elements in the gradient
-    uint64_t first_bucket;   // encode_buckets_kernel: first bucket to handle
+    uint64_t first_bucket;   // first bucket of the plain-load part
     uint64_t num_buckets;    // total buckets of the gradient
     uint64_t num_words;      // total packed words of the gradient
-    uint32_t num_tiles;      // encode_tiles_kernel: full tiles
+    uint32_t num_tiles;      // whole 8192-element tiles taken by the tile path
+    uint32_t plain_ctas;     // the first plain_ctas CTAs run the plain-load part, the rest walk over the tiles
     uint32_t bucket;         // B
-    uint32_t rows_per_tile;  // T / 32
+    uint32_t bucket_log2;    // log2(B) on the tile path
     uint32_t lanes_per_bucket;  // B / 32 when B < 1024, else 32
+    uint32_t warps_per_bucket;  // B / 1024 when B >= 1024, else 1
     float gain_num;          // DQSG: s = (L-1)/2;  NDQSG: A = alpha * M1
-    float shift;             // DQSG: s;  NDQSG: unused
+    float shift;             // DQSG: s
     float kmax;              // DQSG: L - 1
     uint32_t K;              // NDQSG: coarse ratio
     uint32_t K_offset;       // NDQSG any K: multiple of K that is >= 2^22
@@ -39,6 +52,22 @@ struct EncodeArgs {
 };
 
 __device__ unsigned int g_dq_error_flags = 0u;
+
+// Quantize one element to its code.  f = dither + 1.5 in [1, 2).
+template <int MODE>
+__device__ __forceinline__ uint32_t quantize_code(float x, float a, float f, const EncodeArgs& args)
+{
+    const float delta = __fadd_rn(f, -1.5f);                              // exact
+    const float v = __fmaf_rn(x, a, delta);
+    if (MODE == kEncDqsg) {
+        float w = __fadd_rn(v, args.shift);
+        w = fminf(fmaxf(w, 0.0f), args.kmax);                              // clamp, then round: same integer
+        return __float_as_uint(__fadd_rn(w, kMagic)) & 0xFFu;
+    }
+    const uint32_t tb = __float_as_uint(__fadd_rn(v, kMagic));             // kMagicBits + q1 (two's complement)
+    if (MODE == kEncNdqsgPow2) return tb & (args.K - 1u);
+    return (tb - kMagicBits + args.K_offset) % args.K;                     // q1 + positive multiple of K
+}
 
 // Quantize and pack one row.  x: the 32 elements; chunk0: index of the row's first 4-element chunk in the
 // whole gradient (= row index * 8); a: the bucket's gain.  out: the row's BITS words.
@@ -49,33 +78,23 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t chunk0
 #pragma unroll
     for (int j = 0; j < BITS; ++j) out[j] = 0u;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        uint32_t rnd[4];
-        philox4x32_10(chunk0 + (uint32_t)c, args.ps, rnd);
+    for (int h = 0; h < 2; ++h) {                   // four Philox blocks (16 elements) in flight at a time
+        uint32_t ctr[4], rnd[4][4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int idx = 4 * c + e;
-            const float delta = __fadd_rn(dither_f12(rnd[e]), -1.5f);     // exact
-            const float v = __fmaf_rn(x[idx], a, delta);
-            uint32_t code;
-            if (MODE == kEncDqsg) {
-                float w = __fadd_rn(v, args.shift);
-                w = fminf(fmaxf(w, 0.0f), args.kmax);                      // clamp, then round: same integer
-                code = __float_as_uint(__fadd_rn(w, kMagic)) & 0xFFu;
-            } else {
-                const uint32_t tb = __float_as_uint(__fadd_rn(v, kMagic)); // kMagicBits + q1 (two's complement)
-                if (MODE == kEncNdqsgPow2) {
-                    code = tb & (args.K - 1u);
-                } else {
-                    const uint32_t q_off = tb - kMagicBits + args.K_offset; // q1 + multiple of K, positive
-                    code = q_off % args.K;
-                }
+        for (int j = 0; j < 4; ++j) ctr[j] = chunk0 + (uint32_t)(4 * h + j);
+        philox4x32_10_xN<4>(ctr, args.ps, rnd);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int idx = 16 * h + 4 * j + e;
+                const uint32_t code = quantize_code<MODE>(x[idx], a, dither_f12(rnd[j][e]), args);
+                const int bit = idx * BITS;
+                const int wi = bit >> 5;
+                const int sh = bit & 31;
+                out[wi] |= code << sh;
+                if (sh + BITS > 32) out[wi + 1] |= code >> (32 - sh);
             }
-            const int bit = idx * BITS;
-            const int wi = bit >> 5;
-            const int sh = bit & 31;
-            out[wi] |= code << sh;
-            if (sh + BITS > 32) out[wi + 1] |= code >> (32 - sh);
         }
     }
 }
@@ -103,101 +122,11 @@ __device__ __forceinline__ float bucket_gain(float num, float kappa)
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Power-of-two buckets, full tiles.  blockDim.x = 32 * warps; dynamic shared memory =
-// warps * rows_per_tile * 128 + 1024 bytes.
-// ---------------------------------------------------------------------------------------------------
-constexpr int kEncMaxWarps = 8;
-
-template <int BITS, int MODE>
-__global__ void __launch_bounds__(32 * kEncMaxWarps)
-encode_tiles_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ EncodeArgs args)
-{
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[kEncMaxWarps];
-
-    const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t warps = blockDim.x >> 5;
-    const uint32_t tile = blockIdx.x * warps + warp;
-    if (tile >= args.num_tiles) return;
-
-    const uint32_t tile_bytes = args.rows_per_tile * 128u;
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t tile_smem = smem_base + warp * tile_bytes;
-    const uint32_t bar = smem_u32(&bars[warp]);
-    const uint32_t row0 = tile * args.rows_per_tile;        // first row of the tile in the gradient
-
-    if (lane == 0) {
-        mbar_init(bar, 1u);
-        fence_mbar_init();
-    }
-    __syncwarp();
-    if (lane == 0) {
-        mbar_expect_tx(bar, tile_bytes);
-        tma_load_rows(tile_smem, &tmap, bar, (int32_t)row0);
-    }
-    if (!mbar_wait_bounded(bar, 0u)) {
-        if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
-        return;
-    }
-
-    const uint32_t rows_per_lane = args.rows_per_tile >> 5;
-    const uint32_t swz = lane & 7u;                         // (row & 7) is the same for all of a lane's rows
-
-    // pass 1: max |g| over the lane's rows, then over the lanes of the bucket
-    float mx = 0.0f;
-    for (uint32_t k = 0; k < rows_per_lane; ++k) {
-        const uint32_t row_addr = tile_smem + (lane + 32u * k) * 128u;
-#pragma unroll
-        for (uint32_t c = 0; c < 8; ++c) {
-            float4 v;
-            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                         : "r"(row_addr + ((c ^ swz) << 4)));
-            mx = fmaxf(mx, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
-        }
-    }
-    for (uint32_t off = args.lanes_per_bucket >> 1; off > 0; off >>= 1)
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-
-    if (args.bucket >= 1024u) {
-        if (lane == 0) args.scale[tile] = mx;
-    } else if ((lane & (args.lanes_per_bucket - 1u)) == 0u) {
-        const uint32_t buckets_per_tile = 32u / args.lanes_per_bucket;
-        args.scale[(uint64_t)tile * buckets_per_tile + lane / args.lanes_per_bucket] = mx;
-    }
-    const float a = bucket_gain(args.gain_num, mx);
-
-    // pass 2: quantize and pack, one row at a time
-    for (uint32_t k = 0; k < rows_per_lane; ++k) {
-        const uint32_t r = lane + 32u * k;
-        const uint32_t row_addr = tile_smem + r * 128u;
-        float x[32];
-#pragma unroll
-        for (uint32_t c = 0; c < 8; ++c) {
-            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                         : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
-                         : "r"(row_addr + ((c ^ swz) << 4)));
-        }
-        uint32_t out[BITS];
-        const uint32_t grow = row0 + r;
-        encode_row<BITS, MODE>(x, grow * 8u, a, args, out);
-        store_row_words<BITS>(args.packed + (uint64_t)grow * BITS, out);
-    }
-}
-
-// ---------------------------------------------------------------------------------------------------
-// Any bucket size / ragged tail: one warp per bucket, plain loads.
+// Plain-load part: one warp per bucket, any bucket size, ragged end.
 // ---------------------------------------------------------------------------------------------------
 template <int BITS, int MODE>
-__global__ void __launch_bounds__(128)
-encode_buckets_kernel(const __grid_constant__ EncodeArgs args)
+__device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint64_t bucket, uint32_t lane)
 {
-    const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint64_t bucket = args.first_bucket + (uint64_t)blockIdx.x * (blockDim.x >> 5) + warp;
-    if (bucket >= args.num_buckets) return;
-
     const uint64_t lo = bucket * args.bucket;
     const uint32_t len = (uint32_t)((args.n - lo < args.bucket) ? (args.n - lo) : args.bucket);
     const float* g = args.grad + lo;
@@ -241,6 +170,121 @@ encode_buckets_kernel(const __grid_constant__ EncodeArgs args)
                 if (grow * BITS + j < args.num_words) dst[j] = out[j] & m;
             }
         }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// The encode kernel.  Grid = CTAs for the plain-load part (scheduled first) + persistent tile CTAs.
+// Block = 8 consumer warps + 1 producer warp.  Dynamic shared memory = kEncSmemBytes.
+// ---------------------------------------------------------------------------------------------------
+template <int BITS, int MODE>
+__global__ void __launch_bounds__(kEncThreads, 3)
+encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ EncodeArgs args)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kEncStages];
+    __shared__ __align__(8) uint64_t bar_empty[kEncStages];
+    __shared__ float warp_max[2][kConsumerWarps];
+    __shared__ uint32_t s_abort;
+
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t lane = threadIdx.x & 31u;
+
+    if (blockIdx.x < args.plain_ctas) {
+        // plain-load part: consumer warps take buckets round-robin over these CTAs
+        if (warp >= (uint32_t)kConsumerWarps) return;
+        for (uint64_t b = args.first_bucket + (uint64_t)blockIdx.x * kConsumerWarps + warp;
+             b < args.num_buckets; b += (uint64_t)args.plain_ctas * kConsumerWarps)
+            encode_bucket_plain<BITS, MODE>(args, b, lane);
+        return;
+    }
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int s = 0; s < kEncStages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1u);
+            mbar_init(smem_u32(&bar_empty[s]), (uint32_t)kConsumerWarps);
+        }
+        s_abort = 0u;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    const uint32_t stride = gridDim.x - args.plain_ctas;
+    const uint32_t first_tile = blockIdx.x - args.plain_ctas;
+    if (warp == (uint32_t)kConsumerWarps) {
+        // ---------------- producer: keep the ring full
+        if (lane == 0) {
+            uint32_t k = 0;
+            for (uint32_t tile = first_tile; tile < args.num_tiles; tile += stride, ++k) {
+                const uint32_t s = k % kEncStages;
+                const uint32_t use = k / kEncStages;
+                if (use > 0) {
+                    const uint32_t tries = (*(volatile uint32_t*)&s_abort) ? 1u : (1u << 22);
+                    if (!mbar_wait_bounded(smem_u32(&bar_empty[s]), (use - 1u) & 1u, tries)) {
+                        s_abort = 1u;
+                        atomicOr(&g_dq_error_flags, 0x2u);
+                    }
+                }
+                mbar_expect_tx(smem_u32(&bar_full[s]), (uint32_t)kTileBytes);
+                tma_load_rows(smem_base + s * kTileBytes, &tmap, smem_u32(&bar_full[s]),
+                              (int32_t)(tile * kTileRows));
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers
+    const uint32_t swz = lane & 7u;                  // (row & 7): rows are warp*32 + lane
+    const uint32_t row_in_tile = warp * 32u + lane;
+    const uint32_t wpb = args.warps_per_bucket;      // warps sharing a bucket (1, 2, 4, 8)
+    const uint32_t group = warp / wpb;               // bucket of this warp inside the tile, when B >= 1024
+    uint32_t k = 0;
+    for (uint32_t tile = first_tile; tile < args.num_tiles; tile += stride, ++k) {
+        const uint32_t s = k % kEncStages;
+        const uint32_t use = k / kEncStages;
+        {
+            const uint32_t tries = (*(volatile uint32_t*)&s_abort) ? 1u : (1u << 22);
+            if (!mbar_wait_bounded(smem_u32(&bar_full[s]), use & 1u, tries)) {
+                s_abort = 1u;
+                if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
+            }
+        }
+        // the lane's row -> registers, then the stage can be refilled
+        float x[32];
+        const uint32_t row_addr = smem_base + s * kTileBytes + row_in_tile * 128u;
+#pragma unroll
+        for (uint32_t c = 0; c < 8; ++c) {
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                         : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
+                         : "r"(row_addr + ((c ^ swz) << 4))
+                         : "memory");
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
+
+        // max |g| over the bucket
+        float mx = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fabsf(x[e]));
+        for (uint32_t off = args.lanes_per_bucket >> 1; off > 0; off >>= 1)
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+        const uint64_t row = (uint64_t)tile * kTileRows + row_in_tile;   // row index in the gradient
+        if (wpb > 1u) {
+            if (lane == 0) warp_max[k & 1u][warp] = mx;
+            named_bar_sync(1u + group, wpb * 32u);
+            mx = warp_max[k & 1u][group * wpb];
+            for (uint32_t i = 1; i < wpb; ++i) mx = fmaxf(mx, warp_max[k & 1u][group * wpb + i]);
+            if (lane == 0 && (warp % wpb) == 0u) args.scale[(row * 32u) >> args.bucket_log2] = mx;
+        } else if ((lane & (args.lanes_per_bucket - 1u)) == 0u) {
+            args.scale[(row * 32u) >> args.bucket_log2] = mx;
+        }
+        const float a = bucket_gain(args.gain_num, mx);
+
+        uint32_t out[BITS];
+        encode_row<BITS, MODE>(x, (uint32_t)(row * 8u), a, args, out);
+        store_row_words<BITS>(args.packed + row * BITS, out);
     }
 }
 
