@@ -53,47 +53,106 @@ struct EncodeArgs {
 
 __device__ unsigned int g_dq_error_flags = 0u;
 
-// Quantize one element to its code.  f = dither + 1.5 in [1, 2).
-template <int MODE>
-__device__ __forceinline__ uint32_t quantize_code(float x, float a, float f, const EncodeArgs& args)
+// max(m, |a|, |b|) in one instruction (three-input max, sm_100).
+__device__ __forceinline__ float max3_abs(float m, float a, float b)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b)));
+    return d;
+}
+
+// ORs the low `nbits` bits of v into the row's bit stream at bit offset `bit` (all offsets are compile-time).
+template <int BITS>
+__device__ __forceinline__ void put_bits(uint32_t (&out)[BITS], int bit, int nbits, uint32_t v)
+{
+    const int wi = bit >> 5;
+    const int sh = bit & 31;
+    out[wi] |= v << sh;
+    if (sh + nbits > 32) out[wi + 1] |= v >> (32 - sh);
+}
+
+// DQSG: the rounded, clamped index of one element as an exact small float (0 .. L-1).
+//   v = fma(g, a, delta);  w = v + s;  k = clamp(rint(w), 0, L-1)   (clamping before rounding gives the same k)
+// f = dither + 1.5 in [1, 2).
+__device__ __forceinline__ float dqsg_index_f(float x, float a, float f, const EncodeArgs& args)
 {
     const float delta = __fadd_rn(f, -1.5f);                              // exact
     const float v = __fmaf_rn(x, a, delta);
-    if (MODE == kEncDqsg) {
-        float w = __fadd_rn(v, args.shift);
-        w = fminf(fmaxf(w, 0.0f), args.kmax);                              // clamp, then round: same integer
-        return __float_as_uint(__fadd_rn(w, kMagic)) & 0xFFu;
-    }
-    const uint32_t tb = __float_as_uint(__fadd_rn(v, kMagic));             // kMagicBits + q1 (two's complement)
-    if (MODE == kEncNdqsgPow2) return tb & (args.K - 1u);
-    return (tb - kMagicBits + args.K_offset) % args.K;                     // q1 + positive multiple of K
+    float w = __fadd_rn(v, args.shift);
+    w = fminf(fmaxf(w, 0.0f), args.kmax);
+    return __fadd_rn(__fadd_rn(w, kMagic), -kMagic);                      // rint for 0 <= w < 2^22
+}
+
+// NDQSG: bit pattern kMagicBits + q1 (two's complement in the low bits) of one element.
+__device__ __forceinline__ uint32_t ndqsg_index_bits(float x, float a, float f)
+{
+    const float delta = __fadd_rn(f, -1.5f);
+    const float v = __fmaf_rn(x, a, delta);
+    return __float_as_uint(__fadd_rn(v, kMagic));
 }
 
 // Quantize and pack one row.  x: the 32 elements; chunk0: index of the row's first 4-element chunk in the
 // whole gradient (= row index * 8); a: the bucket's gain.  out: the row's BITS words.
+//
+// Integer and logic instructions cost about twice the issue bandwidth of fp32 ones on this GPU, so the DQSG
+// codes are packed in floating point: G = floor(22 / BITS) consecutive indices are combined by exact
+// multiply-adds (sum k_i 2^(BITS i) < 2^22) and only the group is converted and shifted into place.
+// NDQSG codes need their upper bits dropped; when BITS divides 32 that is one shift, and one funnel shift
+// inserts the code.
 template <int BITS, int MODE>
 __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t chunk0, float a,
                                            const EncodeArgs& args, uint32_t (&out)[BITS])
 {
 #pragma unroll
     for (int j = 0; j < BITS; ++j) out[j] = 0u;
+    constexpr int G = 22 / BITS;                    // elements per float group (DQSG)
+    float grp = 0.0f;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {                   // four Philox blocks (16 elements) in flight at a time
         uint32_t ctr[4], rnd[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) ctr[j] = chunk0 + (uint32_t)(4 * h + j);
         philox4x32_10_xN<4>(ctr, args.ps, rnd);
+        if constexpr (MODE == kEncNdqsgPow2 && (32 % BITS) == 0) {
+            // units of U elements (a whole word, or half a word for one bit); elements are inserted from the
+            // last to the first: moving the code to the top of a register drops the bits above it, and one
+            // funnel shift pushes it into the unit.
+            constexpr int U = (32 / BITS < 16) ? (32 / BITS) : 16;
+            uint32_t unit = 0u;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+            for (int j = 3; j >= 0; --j) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int idx = 16 * h + 4 * j + e;
-                const uint32_t code = quantize_code<MODE>(x[idx], a, dither_f12(rnd[j][e]), args);
-                const int bit = idx * BITS;
-                const int wi = bit >> 5;
-                const int sh = bit & 31;
-                out[wi] |= code << sh;
-                if (sh + BITS > 32) out[wi + 1] |= code >> (32 - sh);
+                for (int e = 3; e >= 0; --e) {
+                    const int idx = 16 * h + 4 * j + e;
+                    const uint32_t tb = ndqsg_index_bits(x[idx], a, dither_f12(rnd[j][e]));
+                    unit = __funnelshift_l(tb << (32 - BITS), (idx % U == U - 1) ? 0u : unit, BITS);
+                    if (idx % U == 0) put_bits<BITS>(out, idx * BITS, U * BITS, unit);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int idx = 16 * h + 4 * j + e;
+                    const float f = dither_f12(rnd[j][e]);
+                    if (MODE == kEncDqsg) {
+                        const float kf = dqsg_index_f(x[idx], a, f, args);
+                        const int pos = idx % G;                           // position inside the group
+                        grp = (pos == 0) ? kf : __fmaf_rn(kf, (float)(1u << (BITS * pos)), grp);   // exact
+                        if (pos == G - 1 || idx == 31) {
+                            const int first = idx - pos;
+                            const uint32_t gb = __float_as_uint(__fadd_rn(grp, kMagic)) - kMagicBits;
+                            put_bits<BITS>(out, first * BITS, (pos + 1) * BITS, gb);
+                        }
+                    } else {
+                        const uint32_t tb = ndqsg_index_bits(x[idx], a, f);
+                        uint32_t code;
+                        if (MODE == kEncNdqsgPow2) code = tb & (args.K - 1u);
+                        else code = (tb - kMagicBits + args.K_offset) % args.K;   // q1 + positive multiple of K
+                        put_bits<BITS>(out, idx * BITS, BITS, code);
+                    }
+                }
             }
         }
     }
@@ -267,7 +326,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         // max |g| over the bucket
         float mx = 0.0f;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fabsf(x[e]));
+        for (int e = 0; e < 32; e += 2) mx = max3_abs(mx, x[e], x[e + 1]);
         for (uint32_t off = args.lanes_per_bucket >> 1; off > 0; off >>= 1)
             mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
         const uint64_t row = (uint64_t)tile * kTileRows + row_in_tile;   // row index in the gradient
