@@ -81,6 +81,23 @@ def measured_peaks():
     return 6650.0, "fallback", 1965.0
 
 
+# ------------------------------------------------------------------------------------------ ranks
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_value(step_bytes_per_rank: int, world: int, ms_per_step: float) -> float:
+    """GB/s of the whole job: every rank processes its own replica of the workload (weak scaling)."""
+    return world * step_bytes_per_rank / ms_per_step / 1e6
+
+
 # ------------------------------------------------------------------------------------------ bytes
 def encode_bytes(dq, n, spec, bucket):
     return 4 * n + 4 * dq.packed_words(n, spec.bits) + 4 * dq.num_buckets(n, bucket)
@@ -456,22 +473,16 @@ def main():
     clocks = sampler.stop() if sampler else {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
     assert dq.device_error_flags() == 0, "a kernel reported a copy timeout"
 
-    if world > 1:
-        t = torch.tensor([total_ms, enc_ms, dec_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, enc_ms, dec_ms = (float(x) for x in t.tolist())
+    total_ms, enc_ms, dec_ms = max_over_ranks([total_ms, enc_ms, dec_ms], dev)
     ms_per_step = total_ms / args.steps
     step_bytes = enc_bytes + dec_bytes
-    value = world * step_bytes / ms_per_step / 1e6
+    value = whole_job_value(step_bytes, world, ms_per_step)
 
     kernels = {} if args.no_kernels else kernel_timings(st, hbm_peak, sm_max_mhz)
     e2e = None
     if not args.no_e2e:
         dt, h2d, d2h, _ = run_e2e(st, max(1, min(args.steps, 3)))
-        if world > 1:
-            t = torch.tensor([dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks([dt], dev)[0]
         e2e = {"value": world * step_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3}
 
