@@ -41,7 +41,8 @@ typedef enum {
     DQ_ERR_INVALID_ARG = 1,   /* NULL pointer, n or W out of range, bits/levels/K/alpha out of range      */
     DQ_ERR_UNSUPPORTED = 2,   /* valid in the paper's terms but not handled (e.g. mixed bucket sizes)     */
     DQ_ERR_ALIGNMENT = 3,     /* a device pointer is not 16-byte aligned                                  */
-    DQ_ERR_CUDA = 4           /* a CUDA call or launch failed; see cudaGetLastError of the calling thread */
+    DQ_ERR_CUDA = 4,          /* a CUDA call or launch failed; see cudaGetLastError of the calling thread */
+    DQ_ERR_TOO_LARGE = 5      /* the input does not fit the library's built-in scratch buffer              */
 } dq_status;
 
 typedef enum { DQ_KIND_DQSG = 0, DQ_KIND_NDQSG = 1 } dq_kind;
@@ -142,6 +143,35 @@ dq_status ndqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32
 dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
                                       const float* side_info, float* out_avg,
                                       void* workspace, uint64_t workspace_bytes, void* cuda_stream);
+
+/*
+ * dqsg_encode_host_static -- dqsg_encode_host for callers that cannot provide device memory.
+ * (The paper has no counterpart: this is a packaging variant of the DQSG encoder above.)
+ *
+ * Some users of this library cannot allocate on the GPU at the point where they need to encode: a
+ * training process whose framework has already claimed the device's memory for its own pool, a plug-in
+ * that is only handed host buffers, or a latency-critical loop in which cudaMalloc (which can block and
+ * synchronise the device) is not acceptable.  For them the device-side staging area that dqsg_encode_host
+ * takes as `workspace` lives inside the library instead: a fixed array of DQ_STATIC_SCRATCH_BYTES bytes
+ * in device global memory.  Every GPU on which the library is loaded holds that array until the process
+ * exits, whether or not this function is ever called.
+ *
+ *   grad, out_packed, out_scale   HOST memory, as for dqsg_encode_host (pinned memory keeps the copies
+ *                                 asynchronous); results are complete when the call returns
+ *   returns DQ_ERR_TOO_LARGE      when dq_encode_workspace_bytes(n, p) > DQ_STATIC_SCRATCH_BYTES
+ *                                 (about 7.8 million elements at 2 bits); nothing is copied or launched
+ *
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.  The first call on
+ * each device looks up the array's device address (once per device, with that device current); make that
+ * first call outside any stream capture.  The array is shared by all calls and keeps whatever the last call
+ * left in it.  Nothing in it has to start at zero: the gradient is copied over its input region and the
+ * kernel writes every packed word and every scale before they are copied back.  Two calls that overlap in
+ * time on one device (different host threads or streams) use the same bytes and race; serialise them.
+ */
+#define DQ_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+dq_status dqsg_encode_host_static(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                                  const dq_params* p, uint32_t* out_packed, float* out_scale,
+                                  void* cuda_stream);
 
 /*
  * dq_device_error_flags -- reads (and clears) the current device's error word: DQ_ERR_COPY_TIMEOUT is

@@ -26,6 +26,8 @@ from .binding import (  # noqa: F401
     dqsg_encode_host,
     ndqsg_encode_host,
     ndqsg_decode_aggregate_host,
+    dqsg_encode_host_static,
+    STATIC_SCRATCH_BYTES,
     device_error_flags,
     launch_count,
 )

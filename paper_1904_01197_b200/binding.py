@@ -65,6 +65,8 @@ def lib() -> C.CDLL:
         L.dq_decode_workspace_bytes.argtypes = [pm, u32, u64, C.c_int]; L.dq_decode_workspace_bytes.restype = u64
         for f in (L.dqsg_encode_host, L.ndqsg_encode_host):
             f.argtypes = [vp, u64, u64, u32, u64, pp, vp, vp, vp, u64, vp]; f.restype = C.c_int
+        L.dqsg_encode_host_static.argtypes = [vp, u64, u64, u32, u64, pp, vp, vp, vp]
+        L.dqsg_encode_host_static.restype = C.c_int
         L.ndqsg_decode_aggregate_host.argtypes = [pm, u32, u64, u64, vp, vp, vp, u64, vp]
         L.ndqsg_decode_aggregate_host.restype = C.c_int
         L.dq_device_error_flags.argtypes = [C.POINTER(u32)]; L.dq_device_error_flags.restype = C.c_int
@@ -227,6 +229,22 @@ def dqsg_encode_host(grad, seed, worker, step, params, out_packed, out_scale, wo
 def ndqsg_encode_host(grad, seed, worker, step, params, out_packed, out_scale, workspace, stream=None):
     return _encode_host(lib().ndqsg_encode_host, "ndqsg_encode_host", grad, seed, worker, step, params,
                         out_packed, out_scale, workspace, stream)
+
+
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def dqsg_encode_host_static(grad, seed, worker, step, params, out_packed, out_scale, stream=None):
+    """DQSG encode from host buffers to host buffers without any device allocation by the caller: the
+    staging area is the library's built-in array (at most STATIC_SCRATCH_BYTES for input plus outputs).
+    For callers that cannot allocate GPU memory themselves; calls on one device must not overlap."""
+    n = grad.numel() if isinstance(grad, torch.Tensor) else grad.size
+    _check(lib().dqsg_encode_host_static(_host_ptr(grad, torch.float32, "grad"), n, seed, worker, step,
+                                         C.byref(params), _host_ptr(out_packed, torch.int32, "out_packed"),
+                                         _host_ptr(out_scale, torch.float32, "out_scale"),
+                                         None if stream is None else _stream_ptr(stream)),
+           "dqsg_encode_host_static")
+    return out_packed, out_scale
 
 
 def ndqsg_decode_aggregate_host(msgs: Sequence[Message], n: int, step: int, side_info, out_avg, workspace,

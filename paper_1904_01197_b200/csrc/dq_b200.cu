@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cstring>
+#include <mutex>
 
 #include "dq_decode.cuh"
 #include "dq_encode.cuh"
@@ -301,6 +302,7 @@ const char* dq_status_string(dq_status s)
         case DQ_ERR_UNSUPPORTED: return "unsupported configuration";
         case DQ_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
         case DQ_ERR_CUDA: return "CUDA call failed";
+        case DQ_ERR_TOO_LARGE: return "input larger than the built-in scratch buffer";
     }
     return "unknown status";
 }
@@ -443,6 +445,50 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
     if (cudaMemcpyAsync(out_avg, d_out, n * 4u, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ no allocation
+// Staging area of dqsg_encode_host_static.  In host code this name is only a handle for the runtime, not a
+// device address: the address the kernels and copies use is looked up with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[DQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_scratch_mutex;
+void* g_static_scratch_addr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device; looked up once per device.
+dq_status static_scratch_address(void** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return DQ_ERR_CUDA;
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return DQ_OK;
+}
+}  // namespace
+
+dq_status dqsg_encode_host_static(const float* grad, uint64_t n, uint64_t seed, uint32_t worker, uint64_t step,
+                                  const dq_params* p, uint32_t* out_packed, float* out_scale, void* cuda_stream)
+{
+    uint32_t L;
+    float alpha;
+    dq_status s = check_params(p, DQ_KIND_DQSG, &L, &alpha);
+    if (s != DQ_OK) return s;
+    if (n == 0) return DQ_OK;
+    if (!grad || !out_packed || !out_scale) return DQ_ERR_INVALID_ARG;
+    if (n >= (1ull << 34) || dq_encode_workspace_bytes(n, p) > (uint64_t)DQ_STATIC_SCRATCH_BYTES)
+        return DQ_ERR_TOO_LARGE;
+    void* scratch = nullptr;
+    s = static_scratch_address(&scratch);
+    if (s != DQ_OK) return s;
+    return encode_host(DQ_KIND_DQSG, grad, n, seed, worker, step, p, out_packed, out_scale, scratch,
+                       (uint64_t)DQ_STATIC_SCRATCH_BYTES, cuda_stream);
 }
 
 dq_status dq_device_error_flags(uint32_t* out_flags)
