@@ -197,7 +197,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     }
     a.first_bucket = tiles * (T / B);
     const uint64_t rest = a.num_buckets - a.first_bucket;
-    const uint32_t slots = 3u * (uint32_t)sms;                      // resident CTAs (3 per SM)
+    const uint32_t slots = (uint32_t)dq::kEncCtasPerSm * (uint32_t)sms;   // resident CTAs
     uint32_t plain = 0;
     if (rest > 0) {
         const uint64_t want = (rest + dq::kConsumerWarps - 1u) / dq::kConsumerWarps;

@@ -16,6 +16,11 @@
 
 namespace dq {
 
+#ifndef DQ_DEC_PHILOX_BLOCKS
+#define DQ_DEC_PHILOX_BLOCKS 4
+#endif
+constexpr int kDecPhiloxBlocks = DQ_DEC_PHILOX_BLOCKS;
+
 enum DecKind : uint32_t { kDecDqsg = 0, kDecNdqsgPow2 = 1, kDecNdqsgPow2Shrink = 2, kDecNdqsgAnyK = 3 };
 
 struct DecWorker {
@@ -115,28 +120,29 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
         c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);                 // beta
     }
     const uint32_t chunk0 = (uint32_t)(row * 8u);
+    constexpr int NB = kDecPhiloxBlocks;            // Philox blocks in flight at a time
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        uint32_t ctr[4], rnd[4][4];
+    for (int h = 0; h < 8 / NB; ++h) {
+        uint32_t ctr[NB], rnd[NB][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) ctr[j] = chunk0 + (uint32_t)(4 * h + j);
-        philox4x32_10_xN<4>(ctr, wk.ps, rnd);
+        for (int j = 0; j < NB; ++j) ctr[j] = chunk0 + (uint32_t)(NB * h + j);
+        philox4x32_10_xN<NB>(ctr, wk.ps, rnd);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < NB; ++j) {
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (KIND != kDecDqsg) {
                 if (full_row) {
-                    const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + 4 * h + j);
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + NB * h + j);
                     y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
                 } else {
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        y[e] = (row * 32u + 16u * h + 4u * j + e < n) ? __ldg(side_row + 16 * h + 4 * j + e) : 0.0f;
+                        y[e] = (row * 32u + 4u * (NB * h + j) + e < n) ? __ldg(side_row + 4 * (NB * h + j) + e) : 0.0f;
                 }
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int idx = 16 * h + 4 * j + e;
+                const int idx = 4 * (NB * h + j) + e;
                 const float f = dither_f12(rnd[j][e]);
                 const float X = __fadd_rn(unpack_half_biased<BITS>(words, idx), -wk.cconst);
                 float gt;
@@ -185,8 +191,12 @@ __device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t ro
 }
 
 constexpr int kDecThreads = 128;
+#ifndef DQ_DEC_MINBLOCKS
+#define DQ_DEC_MINBLOCKS 4
+#endif
+constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;
 
-__global__ void __launch_bounds__(kDecThreads, 4)
+__global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
 decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
 {
     const uint64_t row = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;

@@ -129,6 +129,9 @@ __device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap* t
         : "memory");
 }
 
+// Upper bound, in nanoseconds, that one try may stay suspended in hardware before it reports "not yet".
+constexpr uint32_t kWaitHintNs = 20000u;
+
 // Waits for phase `parity` of the barrier; gives up after a fixed number of tries (each try itself blocks
 // for a hardware-defined time), so a copy that never lands cannot hang the kernel.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_tries = (1u << 22))
@@ -137,10 +140,10 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok)
-            : "r"(bar), "r"(parity)
+            : "r"(bar), "r"(parity), "r"(kWaitHintNs)
             : "memory");
         if (ok) return true;
     }

@@ -26,7 +26,14 @@ constexpr int kTileRows = 256;                     // rows per tile (8192 elemen
 constexpr int kTileBytes = kTileRows * 128;
 constexpr int kConsumerWarps = kTileRows / 32;     // one row per lane
 constexpr int kEncThreads = 32 * (kConsumerWarps + 1);
-constexpr int kEncStages = 2;
+#ifndef DQ_ENC_STAGES
+#define DQ_ENC_STAGES 2
+#endif
+#ifndef DQ_ENC_CTAS_PER_SM
+#define DQ_ENC_CTAS_PER_SM 3
+#endif
+constexpr int kEncStages = DQ_ENC_STAGES;
+constexpr int kEncCtasPerSm = DQ_ENC_CTAS_PER_SM;
 constexpr size_t kEncSmemBytes = (size_t)kEncStages * kTileBytes + 1024;
 
 struct EncodeArgs {
@@ -237,7 +244,7 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
 // Block = 8 consumer warps + 1 producer warp.  Dynamic shared memory = kEncSmemBytes.
 // ---------------------------------------------------------------------------------------------------
 template <int BITS, int MODE>
-__global__ void __launch_bounds__(kEncThreads, 3)
+__global__ void __launch_bounds__(kEncThreads, kEncCtasPerSm)
 encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ EncodeArgs args)
 {
     extern __shared__ uint8_t smem_raw[];
