@@ -39,7 +39,8 @@ def build(force: bool = False) -> Path:
 class _Msg(C.Structure):
     _fields_ = [("kind", C.c_uint32), ("bucket", C.c_uint32), ("bits", C.c_uint32),
                 ("levels", C.c_uint32), ("coarse_K", C.c_uint32), ("fine_M", C.c_float),
-                ("alpha", C.c_float), ("worker", C.c_uint32), ("seed", C.c_uint64),
+                ("alpha", C.c_float), ("worker", C.c_uint32), ("dither_bits", C.c_uint32),
+                ("reserved", C.c_uint32), ("seed", C.c_uint64),
                 ("packed", C.c_void_p), ("scale", C.c_void_p)]
 
 
@@ -59,6 +60,12 @@ def lib():
         L.dqo_dither_from_bits.restype = C.c_float
         L.dqo_dither.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint64]
         L.dqo_dither.restype = C.c_float
+        L.dqo_dither16_half.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint64]
+        L.dqo_dither16_half.restype = C.c_uint32
+        L.dqo_dither16_from_half.argtypes = [C.c_uint32]
+        L.dqo_dither16_from_half.restype = C.c_float
+        L.dqo_dither_stream.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint32]
+        L.dqo_dither_stream.restype = C.c_float
         for name, nargs in (("dqo_Q", 2), ("dqo_dithered", 3), ("dqo_nested_encode_scalar", 5),
                             ("dqo_nested_decode_scalar", 5)):
             f = getattr(L, name)
@@ -77,10 +84,10 @@ def lib():
         L.dqo_unpack.argtypes = [u32p, C.c_uint64, C.c_uint32, u32p]
         L.dqo_unpack.restype = None
         L.dqo_dqsg_encode.argtypes = [f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64,
-                                      C.c_uint32, C.c_uint32, C.c_uint32, u32p, f32p, i32p, C.c_int]
+                                      C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, u32p, f32p, i32p, C.c_int]
         L.dqo_dqsg_encode.restype = C.c_int
         L.dqo_ndqsg_encode.argtypes = [f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64,
-                                       C.c_uint32, C.c_uint32, C.c_uint32, C.c_float, C.c_float,
+                                       C.c_uint32, C.c_uint32, C.c_uint32, C.c_float, C.c_float, C.c_uint32,
                                        u32p, f32p, i32p, C.c_int]
         L.dqo_ndqsg_encode.restype = C.c_int
         L.dqo_decode_aggregate.argtypes = [C.POINTER(_Msg), C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64,
@@ -118,9 +125,18 @@ def dither(seed: int, worker: int, step: int, i: int) -> float:
     return float(lib().dqo_dither(seed, worker, step, i))
 
 
-def dither_vector(seed: int, worker: int, step: int, n: int, i0: int = 0) -> np.ndarray:
+def dither_vector(seed: int, worker: int, step: int, n: int, i0: int = 0, dither_bits: int = 32) -> np.ndarray:
     L = lib()
-    return np.array([L.dqo_dither(seed, worker, step, i0 + i) for i in range(n)], dtype=np.float32)
+    return np.array([L.dqo_dither_stream(seed, worker, step, i0 + i, dither_bits) for i in range(n)],
+                    dtype=np.float32)
+
+
+def dither16_half(seed: int, worker: int, step: int, i: int) -> int:
+    return int(lib().dqo_dither16_half(seed, worker, step, i))
+
+
+def dither16_from_half(h: int) -> float:
+    return float(lib().dqo_dither16_from_half(h))
 
 
 def Q(v: float, Delta: float) -> float:
@@ -176,14 +192,14 @@ def _check(rc: int, what: str):
 
 
 def dqsg_encode(g: np.ndarray, seed: int, worker: int, step: int, bucket: int, bits: int,
-                levels: int = 0, i0: int = 0, want_codes: bool = False, threads: int = 1):
+                levels: int = 0, i0: int = 0, want_codes: bool = False, threads: int = 1, dither_bits: int = 32):
     """Returns (packed uint32[NW], scale fp32[NB][, code int32[n]])."""
     g = np.ascontiguousarray(g, dtype=np.float32)
     n = g.size
     packed = np.zeros(max(1, packed_words(n, bits)), dtype=np.uint32)
     scale = np.zeros(max(1, num_buckets(n, bucket)), dtype=np.float32)
     codes = np.zeros(max(1, n), dtype=np.int32) if want_codes else None
-    _check(lib().dqo_dqsg_encode(_p(g, C.c_float), n, i0, seed, worker, step, bucket, bits, levels,
+    _check(lib().dqo_dqsg_encode(_p(g, C.c_float), n, i0, seed, worker, step, bucket, bits, levels, dither_bits,
                                  _p(packed, C.c_uint32), _p(scale, C.c_float), _p(codes, C.c_int32),
                                  threads), "dqsg_encode")
     packed, scale = packed[:packed_words(n, bits)], scale[:num_buckets(n, bucket)]
@@ -192,7 +208,7 @@ def dqsg_encode(g: np.ndarray, seed: int, worker: int, step: int, bucket: int, b
 
 def ndqsg_encode(g: np.ndarray, seed: int, worker: int, step: int, bucket: int, bits: int,
                  coarse_K: int, fine_M: float, alpha: float = 1.0, i0: int = 0,
-                 want_q1: bool = False, threads: int = 1):
+                 want_q1: bool = False, threads: int = 1, dither_bits: int = 32):
     """Returns (packed uint32[NW], scale fp32[NB][, q1 int32[n]])."""
     g = np.ascontiguousarray(g, dtype=np.float32)
     n = g.size
@@ -200,7 +216,7 @@ def ndqsg_encode(g: np.ndarray, seed: int, worker: int, step: int, bucket: int, 
     scale = np.zeros(max(1, num_buckets(n, bucket)), dtype=np.float32)
     q1 = np.zeros(max(1, n), dtype=np.int32) if want_q1 else None
     _check(lib().dqo_ndqsg_encode(_p(g, C.c_float), n, i0, seed, worker, step, bucket, bits, coarse_K,
-                                  fine_M, alpha, _p(packed, C.c_uint32), _p(scale, C.c_float),
+                                  fine_M, alpha, dither_bits, _p(packed, C.c_uint32), _p(scale, C.c_float),
                                   _p(q1, C.c_int32), threads), "ndqsg_encode")
     packed, scale = packed[:packed_words(n, bits)], scale[:num_buckets(n, bucket)]
     return (packed, scale, q1[:n]) if want_q1 else (packed, scale)
@@ -211,12 +227,13 @@ class Msg:
 
     def __init__(self, packed: np.ndarray, scale: np.ndarray, seed: int, worker: int, kind: int,
                  bucket: int, bits: int, levels: int = 0, coarse_K: int = 0, fine_M: float = 0.0,
-                 alpha: float = 1.0):
+                 alpha: float = 1.0, dither_bits: int = 32):
         self.packed = np.ascontiguousarray(packed, dtype=np.uint32)
         self.scale = np.ascontiguousarray(scale, dtype=np.float32)
         self.seed, self.worker, self.kind = seed, worker, kind
         self.bucket, self.bits, self.levels = bucket, bits, levels
         self.coarse_K, self.fine_M, self.alpha = coarse_K, fine_M, alpha
+        self.dither_bits = dither_bits
 
 
 def decode_aggregate(msgs: Sequence[Msg], n: int, step: int, side_info: Optional[np.ndarray] = None,
@@ -226,7 +243,7 @@ def decode_aggregate(msgs: Sequence[Msg], n: int, step: int, side_info: Optional
     arr = (_Msg * max(1, W))()
     for w, m in enumerate(msgs):
         arr[w] = _Msg(m.kind, m.bucket, m.bits, m.levels, m.coarse_K, m.fine_M, m.alpha, m.worker,
-                      m.seed, m.packed.ctypes.data, m.scale.ctypes.data)
+                      m.dither_bits, 0, m.seed, m.packed.ctypes.data, m.scale.ctypes.data)
     if side_info is not None:
         side_info = np.ascontiguousarray(side_info, dtype=np.float32)
         assert side_info.size >= n

@@ -88,6 +88,38 @@ float dqo_dither(uint64_t seed, uint32_t worker, uint64_t step, uint64_t i)
     return dqo_dither_from_bits(dqo_dither_bits(seed, worker, step, i));
 }
 
+/* Second, cheaper stream ("16-bit dither"): one Philox block serves eight elements.  Element i uses block
+ * i/8 (counter = (i/8, worker, step)), word (i mod 8)/2, the low half-word if i is even and the high one if
+ * i is odd.  The 16 bits h give delta = (2h+1) 2^-17 - 1/2: a symmetric grid of 65536 points, never 0 or
+ * +-1/2.  Any uniform pseudo-random sequence over the step serves Algorithm 1; the coarser grid leaves the
+ * error uniform on the step up to 2^-17 of it. */
+uint32_t dqo_dither16_half(uint64_t seed, uint32_t worker, uint64_t step, uint64_t i)
+{
+    uint32_t ctr[4], key[2], out[4];
+    ctr[0] = (uint32_t)(i >> 3);
+    ctr[1] = worker;
+    ctr[2] = (uint32_t)(step & 0xFFFFFFFFu);
+    ctr[3] = (uint32_t)(step >> 32);
+    key[0] = (uint32_t)(seed & 0xFFFFFFFFu);
+    key[1] = (uint32_t)(seed >> 32);
+    dqo_philox4x32_10(ctr, key, out);
+    uint32_t word = out[(i & 7u) >> 1];
+    return (i & 1u) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+float dqo_dither16_from_half(uint32_t h)
+{
+    return (float)(2u * h + 1u) * 0x1p-17f - 0.5f;       /* exact */
+}
+
+/* dither of element i in the stream selected by dither_bits (32: one word per element; 16: see above) */
+float dqo_dither_stream(uint64_t seed, uint32_t worker, uint64_t step, uint64_t i, uint32_t dither_bits)
+{
+    if (dither_bits == 16u)
+        return dqo_dither16_from_half(dqo_dither16_half(seed, worker, step, i));
+    return dqo_dither(seed, worker, step, i);
+}
+
 /* ------------------------------------------------------------------------
  * Scalar definitions in double, the paper's symbols.
  * ---------------------------------------------------------------------- */
@@ -199,11 +231,12 @@ static int check_common(uint32_t bucket, uint32_t bits, uint64_t i0)
  * ---------------------------------------------------------------------- */
 int dqo_dqsg_encode(const float *g, uint64_t n, uint64_t i0,
                     uint64_t seed, uint32_t worker, uint64_t step,
-                    uint32_t bucket, uint32_t bits, uint32_t levels,
+                    uint32_t bucket, uint32_t bits, uint32_t levels, uint32_t dither_bits,
                     uint32_t *packed, float *scale, int32_t *code_out, int threads)
 {
     int rc = check_common(bucket, bits, i0);
     if (rc) return rc;
+    if (dither_bits != 32u && dither_bits != 16u) return DQO_BAD_ARG;
     if (levels == 0u) levels = dqo_default_levels(bits);
     if (levels < 2u || levels > (1u << bits)) return DQO_BAD_ARG;
     uint64_t nb = dqo_num_buckets(n, bucket);
@@ -219,7 +252,7 @@ int dqo_dqsg_encode(const float *g, uint64_t n, uint64_t i0,
         scale[j] = kappa;
         float a = bucket_gain(s, kappa);
         for (uint64_t i = lo; i < lo + len; ++i) {
-            float delta = dqo_dither(seed, worker, step, i0 + i);
+            float delta = dqo_dither_stream(seed, worker, step, i0 + i, dither_bits);
             float v = fmaf(g[i], a, delta);
             float w = v + s;
             int32_t k = (int32_t)rintf(w);
@@ -245,10 +278,11 @@ int dqo_dqsg_encode(const float *g, uint64_t n, uint64_t i0,
 int dqo_ndqsg_encode(const float *g, uint64_t n, uint64_t i0,
                      uint64_t seed, uint32_t worker, uint64_t step,
                      uint32_t bucket, uint32_t bits, uint32_t coarse_K, float fine_M, float alpha,
-                     uint32_t *packed, float *scale, int32_t *q1_out, int threads)
+                     uint32_t dither_bits, uint32_t *packed, float *scale, int32_t *q1_out, int threads)
 {
     int rc = check_common(bucket, bits, i0);
     if (rc) return rc;
+    if (dither_bits != 32u && dither_bits != 16u) return DQO_BAD_ARG;
     if (coarse_K < 2u || coarse_K > (1u << bits)) return DQO_BAD_ARG;
     if (!(fine_M > 0.0f) || !(alpha > 0.0f) || alpha > 1.0f) return DQO_BAD_ARG;
     uint64_t nb = dqo_num_buckets(n, bucket);
@@ -265,7 +299,7 @@ int dqo_ndqsg_encode(const float *g, uint64_t n, uint64_t i0,
         scale[j] = kappa;
         float a = bucket_gain(A, kappa);
         for (uint64_t i = lo; i < lo + len; ++i) {
-            float delta = dqo_dither(seed, worker, step, i0 + i);
+            float delta = dqo_dither_stream(seed, worker, step, i0 + i, dither_bits);
             int32_t q1 = (int32_t)rintf(fmaf(g[i], a, delta));
             int32_t m = ((q1 % K) + K) % K;
             code[i] = (uint32_t)m;
@@ -289,6 +323,8 @@ typedef struct {
     float fine_M;           /* NDQSG */
     float alpha;            /* NDQSG */
     uint32_t worker;
+    uint32_t dither_bits;   /* 32 or 16 */
+    uint32_t reserved;
     uint64_t seed;
     const uint32_t *packed; /* words for elements [i0, i0+n) */
     const float *scale;     /* scales for the same range */
@@ -338,6 +374,7 @@ int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i
         int rc = check_common(m->bucket, m->bits, i0);
         if (rc) return rc;
         if (m->bucket != msgs[0].bucket) return DQO_BAD_ARG;
+        if (m->dither_bits != 32u && m->dither_bits != 16u) return DQO_BAD_ARG;
         if (m->kind == DQO_KIND_DQSG) {
             uint32_t L = m->levels ? m->levels : dqo_default_levels(m->bits);
             if (L < 2u || L > (1u << m->bits)) return DQO_BAD_ARG;
@@ -358,7 +395,7 @@ int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i
         for (uint32_t w = 0; w < W; ++w) {
             const dqo_msg *m = &msgs[w];
             float kappa = m->scale[j];
-            float delta = dqo_dither(m->seed, m->worker, step, i0 + (uint64_t)i);
+            float delta = dqo_dither_stream(m->seed, m->worker, step, i0 + (uint64_t)i, m->dither_bits);
             uint32_t code = dqo_unpack_one(m->packed, (uint64_t)i, m->bits);
             float gt;
             if (m->kind == DQO_KIND_DQSG) {
