@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--workload", default="ndqsg_resnet50",
                     choices=["tiny", "dqsg_resnet18", "ndqsg_resnet50", "ndqsg_gpt2_small"])
     ap.add_argument("--bits", type=int, default=2, help="bits for the dqsg_resnet18 workload (1, 2 or 3)")
+    ap.add_argument("--dither-bits", type=int, default=32, choices=[32, 16],
+                    help="random bits per dither value: 32 (one Philox word per element) or 16 (half a word)")
     ap.add_argument("--n", type=int, default=0, help="override the gradient length (debugging / profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -67,7 +69,7 @@ def make_workload(args, rank: int):
         kw["n"] = args.n
     if args.workload == "dqsg_resnet18":
         kw["bits"] = args.bits
-    return wl.by_name(args.workload, **kw)
+    return wl.by_name(args.workload, dither_bits=args.dither_bits, **kw)
 
 
 def measured_peaks():
@@ -163,7 +165,8 @@ class GpuState:
         from dq_workloads.generators import DQSG
         self.dq, self.torch, self.cfg, self.dev = dq, torch, cfg, dev
         self.DQSG = DQSG
-        self.params = [dq.binding.make_params(cfg.bucket, s.bits, s.levels, s.coarse_K, s.fine_M, s.alpha)
+        self.params = [dq.binding.make_params(cfg.bucket, s.bits, s.levels, s.coarse_K, s.fine_M, s.alpha,
+                                              s.dither_bits)
                        for s in cfg.workers]
         self.grads_host = [torch.from_numpy(cfg.grad(w)).pin_memory() for w in range(cfg.W)]
         self.grads = [g.to(dev, non_blocking=True) for g in self.grads_host]
@@ -331,12 +334,13 @@ def oracle_step(cfg, sample: int, threads: int):
     msgs = []
     for w, s in enumerate(cfg.workers):
         if s.kind == DQSG:
-            pk, sc = oracle.dqsg_encode(grads[w], s.seed, w, cfg.step, cfg.bucket, s.bits, s.levels, threads=threads)
+            pk, sc = oracle.dqsg_encode(grads[w], s.seed, w, cfg.step, cfg.bucket, s.bits, s.levels, threads=threads,
+                                        dither_bits=s.dither_bits)
         else:
             pk, sc = oracle.ndqsg_encode(grads[w], s.seed, w, cfg.step, cfg.bucket, s.bits, s.coarse_K, s.fine_M,
-                                         s.alpha, threads=threads)
+                                         s.alpha, threads=threads, dither_bits=s.dither_bits)
         msgs.append(oracle.Msg(pk, sc, s.seed, w, s.kind, cfg.bucket, s.bits, s.levels, s.coarse_K, s.fine_M,
-                               s.alpha))
+                               s.alpha, s.dither_bits))
     if cfg.side_from_worker0:
         side = oracle.decode_aggregate(msgs[:1], ns, cfg.step, threads=threads)
     any_nd = any(s.kind != DQSG for s in cfg.workers)
@@ -369,7 +373,7 @@ def cpu_baseline(cfg, sample: int):
 
 
 def workload_config(cfg, args):
-    return {"workload": cfg.name, "n": cfg.n, "W": cfg.W, "bucket": cfg.bucket,
+    return {"workload": cfg.name, "n": cfg.n, "W": cfg.W, "bucket": cfg.bucket, "dither_bits": args.dither_bits,
             "workers": sorted({f"{'dqsg' if s.kind == 0 else 'ndqsg'}:b{s.bits}:L{s.levels}:K{s.coarse_K}"
                                for s in cfg.workers}),
             "side_info": "decode of worker 0" if cfg.side_from_worker0 else ("given" if cfg.side_info else "none"),

@@ -13,5 +13,6 @@ from .generators import (  # noqa: F401
     ndqsg_gpt2_small,
     sweep_point,
     by_name,
+    with_dither_bits,
     WORKLOAD_NAMES,
 )

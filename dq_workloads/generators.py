@@ -32,6 +32,7 @@ class WorkerSpec:
     fine_M: float = 0.0       # NDQSG 1/Delta_1 in normalised units
     alpha: float = 1.0        # NDQSG shrinkage
     seed: int = 0             # dither seed shared with the decoder
+    dither_bits: int = 32     # random bits per dither value (32 or 16)
 
 
 @dataclass
@@ -196,6 +197,15 @@ def sweep_point(n: int, W: int, bits: int, bucket: int, kind: str = "dqsg", seed
 WORKLOAD_NAMES = ("tiny", "dqsg_resnet18", "ndqsg_resnet50", "ndqsg_gpt2_small")
 
 
-def by_name(name: str, **kw) -> Workload:
-    return {"tiny": tiny, "dqsg_resnet18": dqsg_resnet18, "ndqsg_resnet50": ndqsg_resnet50,
-            "ndqsg_gpt2_small": ndqsg_gpt2_small}[name](**kw)
+def with_dither_bits(cfg: Workload, dither_bits: int) -> Workload:
+    """The same workload with every worker switched to the given dither stream."""
+    import dataclasses
+    cfg.workers = [dataclasses.replace(s, dither_bits=dither_bits) for s in cfg.workers]
+    cfg.meta = dict(cfg.meta, dither_bits=dither_bits)
+    return cfg
+
+
+def by_name(name: str, dither_bits: int = 32, **kw) -> Workload:
+    cfg = {"tiny": tiny, "dqsg_resnet18": dqsg_resnet18, "ndqsg_resnet50": ndqsg_resnet50,
+           "ndqsg_gpt2_small": ndqsg_gpt2_small}[name](**kw)
+    return with_dither_bits(cfg, dither_bits) if dither_bits != 32 else cfg

@@ -15,8 +15,11 @@
  *     equal partitions, one scale kappa each; the last bucket may be short).
  *   - The dither of element i of worker `worker` at iteration `step` is word (i mod 4) of
  *     Philox4x32-10(key = seed, counter = (i / 4, worker, lo32(step), hi32(step))), mapped to the open
- *     grid {(2j+1) 2^-23 - 1/2} in units of the fine quantization step.  Encoder and decoder must be
- *     given the same (seed, worker, step).
+ *     grid {(2j+1) 2^-23 - 1/2} in units of the fine quantization step.  With dq_params.dither_bits = 16
+ *     one block serves eight elements instead: block i / 8, word (i mod 8) / 2, low half-word for even i
+ *     and high half-word for odd i, mapped to {(2h+1) 2^-17 - 1/2}; this halves the generator's cost,
+ *     which dominates both kernels.  Encoder and decoder must be given the same (seed, worker, step) and
+ *     the same dither_bits.
  *   - A message is `scale` (one fp32 per bucket) plus `packed`: element i's b-bit code at bit offset
  *     i*b of a little-endian stream of 32-bit words; pad bits of the last word are written as 0.
  *   - "device" pointers are CUDA device memory on the current device, 16-byte aligned, owned by the
@@ -61,6 +64,8 @@ typedef struct {
     uint32_t coarse_K;  /* NDQSG: K = Delta_2 / Delta_1, 2..2^b.  Ignored for DQSG.                       */
     float    fine_M;    /* NDQSG: M1 = 1/Delta_1 in units of kappa, 0 < alpha*M1 <= 2^20.                 */
     float    alpha;     /* NDQSG: shrinkage, 0 < alpha <= 1; 0 selects 1.                                 */
+    uint32_t dither_bits; /* random bits per dither value: 32 (0 selects it) or 16, see above              */
+    uint32_t reserved;  /* set to 0                                                                       */
 } dq_params;
 
 /* One worker's message as the decoder sees it. */
@@ -105,8 +110,9 @@ dq_status ndqsg_encode(const float* grad, uint64_t n, uint64_t seed, uint32_t wo
 /*
  * dqsg_decode_aggregate -- server side of Algorithm 1: regenerate every worker's dither, reconstruct
  * g~_w = kappa_w (Delta q_w - u_w) and write the mean over the W workers, summed in array order.
- *   msgs     host array of W messages (1 <= W <= DQ_MAX_WORKERS), all of kind DQSG and of one bucket
- *            size; read during the call, the device buffers they point to are read by the kernel
+ *   msgs     host array of W messages (1 <= W <= DQ_MAX_WORKERS), all of kind DQSG, of one bucket size
+ *            and one dither_bits; read during the call, the device buffers they point to are read by
+ *            the kernel
  *   out_avg  device, fp32[n], fully overwritten
  */
 dq_status dqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,

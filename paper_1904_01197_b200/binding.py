@@ -29,7 +29,8 @@ class DqError(RuntimeError):
 
 class DqParams(C.Structure):
     _fields_ = [("bucket", C.c_uint32), ("bits", C.c_uint32), ("levels", C.c_uint32),
-                ("coarse_K", C.c_uint32), ("fine_M", C.c_float), ("alpha", C.c_float)]
+                ("coarse_K", C.c_uint32), ("fine_M", C.c_float), ("alpha", C.c_float),
+                ("dither_bits", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class DqMsg(C.Structure):
@@ -121,8 +122,8 @@ def _host_ptr(t, dtype, what: str) -> Optional[int]:
 
 
 def make_params(bucket: int, bits: int, levels: int = 0, coarse_K: int = 0, fine_M: float = 0.0,
-                alpha: float = 0.0) -> DqParams:
-    return DqParams(bucket, bits, levels, coarse_K, fine_M, alpha)
+                alpha: float = 0.0, dither_bits: int = 0) -> DqParams:
+    return DqParams(bucket, bits, levels, coarse_K, fine_M, alpha, dither_bits, 0)
 
 
 class Message:

@@ -58,6 +58,7 @@ dq_status check_params(const dq_params* p, dq_kind kind, uint32_t* levels_out, f
     if (!p) return DQ_ERR_INVALID_ARG;
     if (p->bucket < 32u || p->bucket > 65536u || (p->bucket % 32u) != 0u) return DQ_ERR_INVALID_ARG;
     if (p->bits < 1u || p->bits > 8u) return DQ_ERR_INVALID_ARG;
+    if (p->dither_bits != 0u && p->dither_bits != 32u && p->dither_bits != 16u) return DQ_ERR_INVALID_ARG;
     if (kind == DQ_KIND_DQSG) {
         const uint32_t L = p->levels ? p->levels : dq_default_levels(p->bits);
         if (L < 2u || L > (1u << p->bits)) return DQ_ERR_INVALID_ARG;
@@ -110,10 +111,10 @@ bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int MODE, int BITS>
+template <int MODE, int BITS, int DITH>
 cudaError_t launch_encode_one(const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
 {
-    auto k = dq::encode_kernel<BITS, MODE>;
+    auto k = dq::encode_kernel<BITS, MODE, DITH>;
     static thread_local bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dq::kEncSmemBytes);
@@ -124,20 +125,28 @@ cudaError_t launch_encode_one(const CUtensorMap& map, const dq::EncodeArgs& a, u
     return cudaGetLastError();
 }
 
-template <int MODE>
-cudaError_t launch_encode(uint32_t bits, const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid,
-                          cudaStream_t st)
+template <int MODE, int DITH>
+cudaError_t launch_encode_bits(uint32_t bits, const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid,
+                               cudaStream_t st)
 {
     switch (bits) {
-        case 1: return launch_encode_one<MODE, 1>(map, a, grid, st);
-        case 2: return launch_encode_one<MODE, 2>(map, a, grid, st);
-        case 3: return launch_encode_one<MODE, 3>(map, a, grid, st);
-        case 4: return launch_encode_one<MODE, 4>(map, a, grid, st);
-        case 5: return launch_encode_one<MODE, 5>(map, a, grid, st);
-        case 6: return launch_encode_one<MODE, 6>(map, a, grid, st);
-        case 7: return launch_encode_one<MODE, 7>(map, a, grid, st);
-        default: return launch_encode_one<MODE, 8>(map, a, grid, st);
+        case 1: return launch_encode_one<MODE, 1, DITH>(map, a, grid, st);
+        case 2: return launch_encode_one<MODE, 2, DITH>(map, a, grid, st);
+        case 3: return launch_encode_one<MODE, 3, DITH>(map, a, grid, st);
+        case 4: return launch_encode_one<MODE, 4, DITH>(map, a, grid, st);
+        case 5: return launch_encode_one<MODE, 5, DITH>(map, a, grid, st);
+        case 6: return launch_encode_one<MODE, 6, DITH>(map, a, grid, st);
+        case 7: return launch_encode_one<MODE, 7, DITH>(map, a, grid, st);
+        default: return launch_encode_one<MODE, 8, DITH>(map, a, grid, st);
     }
+}
+
+template <int MODE>
+cudaError_t launch_encode(uint32_t bits, bool dither16, const CUtensorMap& map, const dq::EncodeArgs& a,
+                          uint32_t grid, cudaStream_t st)
+{
+    return dither16 ? launch_encode_bits<MODE, 16>(bits, map, a, grid, st)
+                    : launch_encode_bits<MODE, 32>(bits, map, a, grid, st);
 }
 
 dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t seed, uint32_t worker,
@@ -212,9 +221,10 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
         tile_ctas = (uint32_t)(tiles < room ? tiles : room);
     }
     cudaError_t e;
-    if (mode == dq::kEncDqsg) e = launch_encode<dq::kEncDqsg>(p->bits, map, a, plain + tile_ctas, st);
-    else if (mode == dq::kEncNdqsgPow2) e = launch_encode<dq::kEncNdqsgPow2>(p->bits, map, a, plain + tile_ctas, st);
-    else e = launch_encode<dq::kEncNdqsgAnyK>(p->bits, map, a, plain + tile_ctas, st);
+    const bool d16 = (p->dither_bits == 16u);
+    if (mode == dq::kEncDqsg) e = launch_encode<dq::kEncDqsg>(p->bits, d16, map, a, plain + tile_ctas, st);
+    else if (mode == dq::kEncNdqsgPow2) e = launch_encode<dq::kEncNdqsgPow2>(p->bits, d16, map, a, plain + tile_ctas, st);
+    else e = launch_encode<dq::kEncNdqsgAnyK>(p->bits, d16, map, a, plain + tile_ctas, st);
     if (e != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;
@@ -235,6 +245,7 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         if (s != DQ_OK) return s;
         if (m.kind == DQ_KIND_NDQSG && !allow_nested) return DQ_ERR_INVALID_ARG;
         if (m.p.bucket != msgs[0].p.bucket) return DQ_ERR_UNSUPPORTED;
+        if ((m.p.dither_bits == 16u) != (msgs[0].p.dither_bits == 16u)) return DQ_ERR_UNSUPPORTED;
         dq::DecWorker& d = a.w[w];
         d.packed = m.packed;
         d.scale = m.scale;
@@ -278,7 +289,8 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
     const uint64_t grid64 = (a.rows + dq::kDecThreads - 1u) / dq::kDecThreads;
     if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
-    dq::decode_aggregate_kernel<<<(uint32_t)grid64, dq::kDecThreads, 0, st>>>(a);
+    if (msgs[0].p.dither_bits == 16u) dq::decode_aggregate_kernel<16><<<(uint32_t)grid64, dq::kDecThreads, 0, st>>>(a);
+    else dq::decode_aggregate_kernel<32><<<(uint32_t)grid64, dq::kDecThreads, 0, st>>>(a);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;

@@ -16,11 +16,6 @@
 
 namespace dq {
 
-#ifndef DQ_DEC_PHILOX_BLOCKS
-#define DQ_DEC_PHILOX_BLOCKS 4
-#endif
-constexpr int kDecPhiloxBlocks = DQ_DEC_PHILOX_BLOCKS;
-
 enum DecKind : uint32_t { kDecDqsg = 0, kDecNdqsgPow2 = 1, kDecNdqsgPow2Shrink = 2, kDecNdqsgAnyK = 3 };
 
 struct DecWorker {
@@ -101,7 +96,7 @@ __device__ __forceinline__ void load_row_words(const uint32_t* src, bool full_ro
 // One worker's contribution to the 32 accumulators of a row.
 //   DQSG:  g~ = (kappa/s) ((k - s) - delta); (k - s + 1.5) - f rounds once to the same value.
 //   NDQSG: r = (m - delta) - y a;  jj = rint(r / K);  q1^ = m - K jj;  g~ = beta (q1^ - delta) [+ (1-alpha^2) y]
-template <int BITS, uint32_t KIND>
+template <int BITS, uint32_t KIND, int DITH>
 __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
                                            uint64_t n, const float* __restrict__ side_row, float (&acc)[32],
                                            uint32_t* status)
@@ -119,31 +114,32 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
         a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
         c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);                 // beta
     }
-    const uint32_t chunk0 = (uint32_t)(row * 8u);
-    constexpr int NB = kDecPhiloxBlocks;            // Philox blocks in flight at a time
+    constexpr int EPB = (DITH == 16) ? 8 : 4;       // elements per Philox block
+    constexpr int PASS = 4 * EPB;                   // elements per group of four blocks
 #pragma unroll
-    for (int h = 0; h < 8 / NB; ++h) {
-        uint32_t ctr[NB], rnd[NB][4];
+    for (int h = 0; h < 32 / PASS; ++h) {
+        uint32_t ctr[4], rnd[4][4];
 #pragma unroll
-        for (int j = 0; j < NB; ++j) ctr[j] = chunk0 + (uint32_t)(NB * h + j);
-        philox4x32_10_xN<NB>(ctr, wk.ps, rnd);
+        for (int j = 0; j < 4; ++j) ctr[j] = (uint32_t)row * (32u / EPB) + (uint32_t)(4 * h + j);
+        philox4x32_10_xN<4>(ctr, wk.ps, rnd);
 #pragma unroll
-        for (int j = 0; j < NB; ++j) {
+        for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (KIND != kDecDqsg) {
                 if (full_row) {
-                    const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + NB * h + j);
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + (PASS / 4) * h + q);
                     y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
                 } else {
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        y[e] = (row * 32u + 4u * (NB * h + j) + e < n) ? __ldg(side_row + 4 * (NB * h + j) + e) : 0.0f;
+                        y[e] = (row * 32u + PASS * h + 4u * q + e < n) ? __ldg(side_row + PASS * h + 4 * q + e) : 0.0f;
                 }
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int idx = 4 * (NB * h + j) + e;
-                const float f = dither_f12(rnd[j][e]);
+                const int t = 4 * q + e;
+                const int idx = PASS * h + t;
+                const float f = dither_of<DITH>(rnd, t);
                 const float X = __fadd_rn(unpack_half_biased<BITS>(words, idx), -wk.cconst);
                 float gt;
                 if (KIND == kDecDqsg) {
@@ -173,20 +169,20 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
     }
 }
 
-template <uint32_t KIND>
+template <uint32_t KIND, int DITH>
 __device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
                                                 uint64_t n, const float* side_row, float (&acc)[32],
                                                 uint32_t* status)
 {
     switch (wk.bits) {
-        case 1: decode_row<1, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 2: decode_row<2, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 3: decode_row<3, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 4: decode_row<4, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 5: decode_row<5, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 6: decode_row<6, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 7: decode_row<7, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        default: decode_row<8, KIND>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 1: decode_row<1, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 2: decode_row<2, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 3: decode_row<3, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 4: decode_row<4, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 5: decode_row<5, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 6: decode_row<6, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 7: decode_row<7, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        default: decode_row<8, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
     }
 }
 
@@ -196,6 +192,7 @@ constexpr int kDecThreads = 128;
 #endif
 constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;
 
+template <int DITH>
 __global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
 decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
 {
@@ -214,10 +211,10 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     for (uint32_t w = 0; w < args.W; ++w) {
         const DecWorker& wk = args.w[w];
         switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
-            default: decode_row_bits<kDecNdqsgAnyK>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            case kDecDqsg: decode_row_bits<kDecDqsg, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            default: decode_row_bits<kDecNdqsgAnyK, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
         }
     }
 

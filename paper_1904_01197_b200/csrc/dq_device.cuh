@@ -92,6 +92,21 @@ __device__ __forceinline__ float dither_f12(uint32_t x)
     return __uint_as_float((x >> 9) | 0x3F800001u);
 }
 
+// 16-bit stream: half-word h -> f = 1 + (2h+1) 2^-17 in [1, 2); the dither is again f - 1.5 (exact).
+__device__ __forceinline__ float dither16_f12(uint32_t word, int high)
+{
+    const uint32_t v = high ? (word >> 9) : (word << 7);
+    return __uint_as_float((v & 0x007FFF80u) | 0x3F800040u);
+}
+
+// f of element t (0 .. 4*EPB-1) of a group of four Philox blocks; EPB = elements per block (4 or 8).
+template <int DITH>
+__device__ __forceinline__ float dither_of(const uint32_t (&rnd)[4][4], int t)
+{
+    if (DITH == 16) return dither16_f12(rnd[t >> 3][(t & 7) >> 1], t & 1);
+    return dither_f12(rnd[t >> 2][t & 3]);
+}
+
 // Round-to-nearest-even of |w| < 2^22 by adding 1.5 * 2^23: the integer lands in the low mantissa bits.
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr uint32_t kMagicBits = 0x4B400000u;   // bit pattern of kMagic

@@ -98,27 +98,30 @@ __device__ __forceinline__ uint32_t ndqsg_index_bits(float x, float a, float f)
     return __float_as_uint(__fadd_rn(v, kMagic));
 }
 
-// Quantize and pack one row.  x: the 32 elements; chunk0: index of the row's first 4-element chunk in the
-// whole gradient (= row index * 8); a: the bucket's gain.  out: the row's BITS words.
+// Quantize and pack one row.  x: the 32 elements; row: index of the row in the whole gradient (the Philox
+// counters follow from it); a: the bucket's gain.  out: the row's BITS words.  DITH: 32 or 16 random bits
+// per dither value.
 //
 // Integer and logic instructions cost about twice the issue bandwidth of fp32 ones on this GPU, so the DQSG
 // codes are packed in floating point: G = floor(22 / BITS) consecutive indices are combined by exact
 // multiply-adds (sum k_i 2^(BITS i) < 2^22) and only the group is converted and shifted into place.
 // NDQSG codes need their upper bits dropped; when BITS divides 32 that is one shift, and one funnel shift
 // inserts the code.
-template <int BITS, int MODE>
-__device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t chunk0, float a,
+template <int BITS, int MODE, int DITH>
+__device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, float a,
                                            const EncodeArgs& args, uint32_t (&out)[BITS])
 {
 #pragma unroll
     for (int j = 0; j < BITS; ++j) out[j] = 0u;
     constexpr int G = 22 / BITS;                    // elements per float group (DQSG)
+    constexpr int EPB = (DITH == 16) ? 8 : 4;       // elements per Philox block
+    constexpr int PASS = 4 * EPB;                   // elements per group of four blocks
     float grp = 0.0f;
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {                   // four Philox blocks (16 elements) in flight at a time
+    for (int h = 0; h < 32 / PASS; ++h) {           // four Philox blocks in flight at a time
         uint32_t ctr[4], rnd[4][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) ctr[j] = chunk0 + (uint32_t)(4 * h + j);
+        for (int j = 0; j < 4; ++j) ctr[j] = row * (32u / EPB) + (uint32_t)(4 * h + j);
         philox4x32_10_xN<4>(ctr, args.ps, rnd);
         if constexpr (MODE == kEncNdqsgPow2 && (32 % BITS) == 0) {
             // units of U elements (a whole word, or half a word for one bit); elements are inserted from the
@@ -127,38 +130,32 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t chunk0
             constexpr int U = (32 / BITS < 16) ? (32 / BITS) : 16;
             uint32_t unit = 0u;
 #pragma unroll
-            for (int j = 3; j >= 0; --j) {
-#pragma unroll
-                for (int e = 3; e >= 0; --e) {
-                    const int idx = 16 * h + 4 * j + e;
-                    const uint32_t tb = ndqsg_index_bits(x[idx], a, dither_f12(rnd[j][e]));
-                    unit = __funnelshift_l(tb << (32 - BITS), (idx % U == U - 1) ? 0u : unit, BITS);
-                    if (idx % U == 0) put_bits<BITS>(out, idx * BITS, U * BITS, unit);
-                }
+            for (int t = PASS - 1; t >= 0; --t) {
+                const int idx = PASS * h + t;
+                const uint32_t tb = ndqsg_index_bits(x[idx], a, dither_of<DITH>(rnd, t));
+                unit = __funnelshift_l(tb << (32 - BITS), (idx % U == U - 1) ? 0u : unit, BITS);
+                if (idx % U == 0) put_bits<BITS>(out, idx * BITS, U * BITS, unit);
             }
         } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int idx = 16 * h + 4 * j + e;
-                    const float f = dither_f12(rnd[j][e]);
-                    if (MODE == kEncDqsg) {
-                        const float kf = dqsg_index_f(x[idx], a, f, args);
-                        const int pos = idx % G;                           // position inside the group
-                        grp = (pos == 0) ? kf : __fmaf_rn(kf, (float)(1u << (BITS * pos)), grp);   // exact
-                        if (pos == G - 1 || idx == 31) {
-                            const int first = idx - pos;
-                            const uint32_t gb = __float_as_uint(__fadd_rn(grp, kMagic)) - kMagicBits;
-                            put_bits<BITS>(out, first * BITS, (pos + 1) * BITS, gb);
-                        }
-                    } else {
-                        const uint32_t tb = ndqsg_index_bits(x[idx], a, f);
-                        uint32_t code;
-                        if (MODE == kEncNdqsgPow2) code = tb & (args.K - 1u);
-                        else code = (tb - kMagicBits + args.K_offset) % args.K;   // q1 + positive multiple of K
-                        put_bits<BITS>(out, idx * BITS, BITS, code);
+            for (int t = 0; t < PASS; ++t) {
+                const int idx = PASS * h + t;
+                const float f = dither_of<DITH>(rnd, t);
+                if (MODE == kEncDqsg) {
+                    const float kf = dqsg_index_f(x[idx], a, f, args);
+                    const int pos = idx % G;                               // position inside the group
+                    grp = (pos == 0) ? kf : __fmaf_rn(kf, (float)(1u << (BITS * pos)), grp);   // exact
+                    if (pos == G - 1 || idx == 31) {
+                        const int first = idx - pos;
+                        const uint32_t gb = __float_as_uint(__fadd_rn(grp, kMagic)) - kMagicBits;
+                        put_bits<BITS>(out, first * BITS, (pos + 1) * BITS, gb);
                     }
+                } else {
+                    const uint32_t tb = ndqsg_index_bits(x[idx], a, f);
+                    uint32_t code;
+                    if (MODE == kEncNdqsgPow2) code = tb & (args.K - 1u);
+                    else code = (tb - kMagicBits + args.K_offset) % args.K;   // q1 + positive multiple of K
+                    put_bits<BITS>(out, idx * BITS, BITS, code);
                 }
             }
         }
@@ -190,7 +187,7 @@ __device__ __forceinline__ float bucket_gain(float num, float kappa)
 // ---------------------------------------------------------------------------------------------------
 // Plain-load part: one warp per bucket, any bucket size, ragged end.
 // ---------------------------------------------------------------------------------------------------
-template <int BITS, int MODE>
+template <int BITS, int MODE, int DITH>
 __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint64_t bucket, uint32_t lane)
 {
     const uint64_t lo = bucket * args.bucket;
@@ -221,7 +218,7 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
         }
         uint32_t out[BITS];
         const uint64_t grow = (lo >> 5) + r;
-        encode_row<BITS, MODE>(x, (uint32_t)(grow * 8u), a, args, out);
+        encode_row<BITS, MODE, DITH>(x, (uint32_t)grow, a, args, out);
         uint32_t* dst = args.packed + grow * BITS;
         if (nvalid == 32u) {
             store_row_words<BITS>(dst, out);
@@ -243,7 +240,7 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
 // The encode kernel.  Grid = CTAs for the plain-load part (scheduled first) + persistent tile CTAs.
 // Block = 8 consumer warps + 1 producer warp.  Dynamic shared memory = kEncSmemBytes.
 // ---------------------------------------------------------------------------------------------------
-template <int BITS, int MODE>
+template <int BITS, int MODE, int DITH>
 __global__ void __launch_bounds__(kEncThreads, kEncCtasPerSm)
 encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ EncodeArgs args)
 {
@@ -261,7 +258,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         if (warp >= (uint32_t)kConsumerWarps) return;
         for (uint64_t b = args.first_bucket + (uint64_t)blockIdx.x * kConsumerWarps + warp;
              b < args.num_buckets; b += (uint64_t)args.plain_ctas * kConsumerWarps)
-            encode_bucket_plain<BITS, MODE>(args, b, lane);
+            encode_bucket_plain<BITS, MODE, DITH>(args, b, lane);
         return;
     }
 
@@ -349,7 +346,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         const float a = bucket_gain(args.gain_num, mx);
 
         uint32_t out[BITS];
-        encode_row<BITS, MODE>(x, (uint32_t)(row * 8u), a, args, out);
+        encode_row<BITS, MODE, DITH>(x, (uint32_t)row, a, args, out);
         store_row_words<BITS>(args.packed + row * BITS, out);
     }
 }

@@ -9,7 +9,8 @@ from dq_workloads.generators import DQSG, NDQSG, WorkerSpec
 
 
 def spec_params(dq, spec: WorkerSpec, bucket: int):
-    return dq.binding.make_params(bucket, spec.bits, spec.levels, spec.coarse_K, spec.fine_M, spec.alpha)
+    return dq.binding.make_params(bucket, spec.bits, spec.levels, spec.coarse_K, spec.fine_M, spec.alpha,
+                                  spec.dither_bits)
 
 
 def gpu_encode(dq, torch, g_dev, spec: WorkerSpec, worker: int, step: int, bucket: int):
@@ -24,14 +25,14 @@ def oracle_encode(oracle, g: np.ndarray, spec: WorkerSpec, worker: int, step: in
                   threads: int = 4):
     if spec.kind == DQSG:
         return oracle.dqsg_encode(g, spec.seed, worker, step, bucket, spec.bits, spec.levels, i0=i0,
-                                  threads=threads)
+                                  threads=threads, dither_bits=spec.dither_bits)
     return oracle.ndqsg_encode(g, spec.seed, worker, step, bucket, spec.bits, spec.coarse_K, spec.fine_M,
-                               spec.alpha, i0=i0, threads=threads)
+                               spec.alpha, i0=i0, threads=threads, dither_bits=spec.dither_bits)
 
 
 def oracle_msg(oracle, packed, scale, spec: WorkerSpec, worker: int, bucket: int):
     return oracle.Msg(packed, scale, spec.seed, worker, spec.kind, bucket, spec.bits, spec.levels,
-                      spec.coarse_K, spec.fine_M, spec.alpha)
+                      spec.coarse_K, spec.fine_M, spec.alpha, spec.dither_bits)
 
 
 def gpu_msg(dq, packed_dev, scale_dev, spec: WorkerSpec, worker: int, bucket: int):

@@ -34,8 +34,8 @@ def test_library_exports_every_declared_symbol(dq):
 
 
 def test_struct_layout_matches_header(dq):
-    assert C.sizeof(dq.DqParams) == 24
-    assert C.sizeof(dq.DqMsg) == 56
+    assert C.sizeof(dq.DqParams) == 32
+    assert C.sizeof(dq.DqMsg) == 64
     assert dq.DqMsg.p.offset == 32 and dq.DqMsg.seed.offset == 16
 
 
@@ -61,6 +61,7 @@ def test_invalid_arguments_are_rejected_before_any_launch(dq):
         (P(512, 9), 1),
         (P(512, 2, 5), 1),                             # 5 levels do not fit 2 bits
         (P(512, 2, 1), 1),                             # one level
+        (P(512, 2, 3, dither_bits=8), 1),              # unknown dither stream
     ]
     for p, want in bad:
         assert L.dqsg_encode(fake, 1024, 1, 0, 0, C.byref(p), fake, fake, None) == want
@@ -93,6 +94,9 @@ def test_invalid_arguments_are_rejected_before_any_launch(dq):
     other = dq.DqMsg(fake, fake, 1, 0, dq.DQ_KIND_DQSG, P(1024, 2))
     arr3 = (dq.DqMsg * 2)(m, other)
     assert L.dqsg_decode_aggregate(arr3, 2, 1024, 0, fake, None) == 2                     # mixed bucket sizes
+    d16 = dq.DqMsg(fake, fake, 1, 0, dq.DQ_KIND_DQSG, P(512, 2, dither_bits=16))
+    arr4 = (dq.DqMsg * 2)(m, d16)
+    assert L.dqsg_decode_aggregate(arr4, 2, 1024, 0, fake, None) == 2                     # mixed dither streams
     assert L.dqsg_decode_aggregate(arr, 2, 0, 0, fake, None) == 0                         # n = 0
     assert L.dq_launch_count() == 0
 
