@@ -196,7 +196,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     CUtensorMap map;
     std::memset(&map, 0, sizeof(map));
     if (tiles > 0) {
-        if (!make_row_map(&map, grad, tiles * dq::kTileRows, dq::kTileRows)) return DQ_ERR_CUDA;
+        if (!make_row_map(&map, grad, tiles * dq::kTileRows, 32u)) return DQ_ERR_CUDA;
         a.num_tiles = (uint32_t)tiles;
         a.lanes_per_bucket = (B < 1024u) ? (B / 32u) : 32u;
         a.warps_per_bucket = (B < 1024u) ? 1u : (B / 1024u);

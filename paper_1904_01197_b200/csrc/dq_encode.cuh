@@ -5,12 +5,12 @@
 // `bits` 32-bit words of the bit stream.  One lane quantizes and packs a whole row, so no lane ever shares a
 // packed word with another lane and no shuffles are needed for packing.
 //
-// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight consumer warps plus one
-// producer warp walk over tiles of 8192 elements (256 rows).  The producer keeps a ring of shared-memory
-// stages filled with asynchronous 2-D tile copies (128-byte swizzle, which makes "lane r reads row r" free of
-// bank conflicts).  A consumer warp takes its 32 rows of a stage into registers, hands the stage back at
-// once, reduces max|g| over its bucket (shuffles inside the warp, a named barrier between the warps that
-// share a bucket) and then quantizes from registers.  The gradient is read from HBM exactly once.
+// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight warps walk over tiles of 8192
+// elements (256 rows).  Every warp owns 32 rows of each tile and keeps its own two-stage shared-memory
+// pipeline filled with asynchronous 2-D tile copies (128-byte swizzle, which makes "lane r reads row r" free
+// of bank conflicts): it takes its rows of a stage into registers, re-arms the stage with the copy for the
+// tile after next, reduces max|g| over its bucket (shuffles inside the warp, a named barrier between the
+// warps that share a bucket) and then quantizes from registers.  The gradient is read from HBM exactly once.
 //
 // Everything else -- other bucket sizes, the part of the vector past the last whole tile, the ragged end --
 // is handled by plain-load code, one warp per bucket, in extra CTAs of the same launch.
@@ -25,7 +25,8 @@ enum EncMode : int { kEncDqsg = 0, kEncNdqsgPow2 = 1, kEncNdqsgAnyK = 2 };
 constexpr int kTileRows = 256;                     // rows per tile (8192 elements, 32 KB)
 constexpr int kTileBytes = kTileRows * 128;
 constexpr int kConsumerWarps = kTileRows / 32;     // one row per lane
-constexpr int kEncThreads = 32 * (kConsumerWarps + 1);
+constexpr int kWarpTileBytes = 32 * 128;           // the 32 rows of a tile that one warp owns
+constexpr int kEncThreads = 32 * kConsumerWarps;
 #ifndef DQ_ENC_STAGES
 #define DQ_ENC_STAGES 2
 #endif
@@ -238,24 +239,26 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
 
 // ---------------------------------------------------------------------------------------------------
 // The encode kernel.  Grid = CTAs for the plain-load part (scheduled first) + persistent tile CTAs.
-// Block = 8 consumer warps + 1 producer warp.  Dynamic shared memory = kEncSmemBytes.
+// Block = 8 warps.  Dynamic shared memory = kEncSmemBytes.
+//
+// Tile path: a CTA walks over tiles of 8192 elements; warp w owns rows [32 w, 32 w + 32) of each tile and
+// runs its own two-stage pipeline: its lane 0 issues the 4 KB tile copy for the tile after next as soon as
+// the warp has taken the current rows into registers, so a copy is always in flight while the warp
+// quantizes, and no warp ever waits for another one except the warps that share a bucket (named barrier).
 // ---------------------------------------------------------------------------------------------------
 template <int BITS, int MODE, int DITH>
 __global__ void __launch_bounds__(kEncThreads, kEncCtasPerSm)
 encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ EncodeArgs args)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[kEncStages];
-    __shared__ __align__(8) uint64_t bar_empty[kEncStages];
+    __shared__ __align__(8) uint64_t bar_full[kConsumerWarps][kEncStages];
     __shared__ float warp_max[2][kConsumerWarps];
-    __shared__ uint32_t s_abort;
 
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31u;
 
     if (blockIdx.x < args.plain_ctas) {
-        // plain-load part: consumer warps take buckets round-robin over these CTAs
-        if (warp >= (uint32_t)kConsumerWarps) return;
+        // plain-load part: warps take buckets round-robin over these CTAs
         for (uint64_t b = args.first_bucket + (uint64_t)blockIdx.x * kConsumerWarps + warp;
              b < args.num_buckets; b += (uint64_t)args.plain_ctas * kConsumerWarps)
             encode_bucket_plain<BITS, MODE, DITH>(args, b, lane);
@@ -263,60 +266,42 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     }
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int s = 0; s < kEncStages; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1u);
-            mbar_init(smem_u32(&bar_empty[s]), (uint32_t)kConsumerWarps);
-        }
-        s_abort = 0u;
-        fence_mbar_init();
-    }
-    __syncthreads();
-
+    const uint32_t my_smem = smem_base + warp * (uint32_t)(kEncStages * kWarpTileBytes);
+    const uint32_t my_bar = smem_u32(&bar_full[warp][0]);
     const uint32_t stride = gridDim.x - args.plain_ctas;
     const uint32_t first_tile = blockIdx.x - args.plain_ctas;
-    if (warp == (uint32_t)kConsumerWarps) {
-        // ---------------- producer: keep the ring full
-        if (lane == 0) {
-            uint32_t k = 0;
-            for (uint32_t tile = first_tile; tile < args.num_tiles; tile += stride, ++k) {
-                const uint32_t s = k % kEncStages;
-                const uint32_t use = k / kEncStages;
-                if (use > 0) {
-                    const uint32_t tries = (*(volatile uint32_t*)&s_abort) ? 1u : (1u << 22);
-                    if (!mbar_wait_bounded(smem_u32(&bar_empty[s]), (use - 1u) & 1u, tries)) {
-                        s_abort = 1u;
-                        atomicOr(&g_dq_error_flags, 0x2u);
-                    }
-                }
-                mbar_expect_tx(smem_u32(&bar_full[s]), (uint32_t)kTileBytes);
-                tma_load_rows(smem_base + s * kTileBytes, &tmap, smem_u32(&bar_full[s]),
-                              (int32_t)(tile * kTileRows));
+
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kEncStages; ++s) mbar_init(my_bar + 8u * s, 1u);
+        fence_mbar_init();
+#pragma unroll
+        for (int s = 0; s < kEncStages; ++s) {
+            const uint64_t tile = (uint64_t)first_tile + (uint64_t)s * stride;
+            if (tile < args.num_tiles) {
+                mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
+                tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
+                              (int32_t)(tile * kTileRows + warp * 32u));
             }
         }
-        return;
     }
+    __syncwarp();
 
-    // ---------------- consumers
-    const uint32_t swz = lane & 7u;                  // (row & 7): rows are warp*32 + lane
-    const uint32_t row_in_tile = warp * 32u + lane;
+    const uint32_t swz = lane & 7u;                  // (row & 7): the warp's rows start at a multiple of 32
     const uint32_t wpb = args.warps_per_bucket;      // warps sharing a bucket (1, 2, 4, 8)
     const uint32_t group = warp / wpb;               // bucket of this warp inside the tile, when B >= 1024
+    bool gave_up = false;
     uint32_t k = 0;
-    for (uint32_t tile = first_tile; tile < args.num_tiles; tile += stride, ++k) {
+    for (uint64_t tile = first_tile; tile < args.num_tiles; tile += stride, ++k) {
         const uint32_t s = k % kEncStages;
         const uint32_t use = k / kEncStages;
-        {
-            const uint32_t tries = (*(volatile uint32_t*)&s_abort) ? 1u : (1u << 22);
-            if (!mbar_wait_bounded(smem_u32(&bar_full[s]), use & 1u, tries)) {
-                s_abort = 1u;
-                if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
-            }
+        if (!mbar_wait_bounded(my_bar + 8u * s, use & 1u, gave_up ? 1u : (1u << 22))) {
+            gave_up = true;
+            if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
         }
-        // the lane's row -> registers, then the stage can be refilled
+        // the lane's row -> registers
         float x[32];
-        const uint32_t row_addr = smem_base + s * kTileBytes + row_in_tile * 128u;
+        const uint32_t row_addr = my_smem + s * kWarpTileBytes + lane * 128u;
 #pragma unroll
         for (uint32_t c = 0; c < 8; ++c) {
             asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
@@ -324,16 +309,23 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                          : "r"(row_addr + ((c ^ swz) << 4))
                          : "memory");
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
-
-        // max |g| over the bucket
+        // max |g| over the bucket.  Every lane has used all of its loaded values once it reaches the
+        // __syncwarp below, so after it the stage can be overwritten by the next copy.
         float mx = 0.0f;
 #pragma unroll
         for (int e = 0; e < 32; e += 2) mx = max3_abs(mx, x[e], x[e + 1]);
         for (uint32_t off = args.lanes_per_bucket >> 1; off > 0; off >>= 1)
             mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-        const uint64_t row = (uint64_t)tile * kTileRows + row_in_tile;   // row index in the gradient
+        __syncwarp();
+        if (lane == 0) {
+            const uint64_t next = tile + (uint64_t)kEncStages * stride;
+            if (next < args.num_tiles) {
+                mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
+                tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
+                              (int32_t)(next * kTileRows + warp * 32u));
+            }
+        }
+        const uint64_t row = tile * kTileRows + warp * 32u + lane;       // row index in the gradient
         if (wpb > 1u) {
             if (lane == 0) warp_max[k & 1u][warp] = mx;
             named_bar_sync(1u + group, wpb * 32u);
