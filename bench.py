@@ -36,6 +36,12 @@ METRIC = "encode / fused decode-aggregate GB/s and % of HBM peak on 1 B200; Gele
 L2_BYTES = 126 * 1024 * 1024
 HBM_NOMINAL_GBS = 8000.0
 SM_COUNT, ISSUE_PER_SM_CLK, LANES = 148, 4, 32           # ALU-issue ceiling: SMs x schedulers x lanes x clock
+# Algorithmic lane-instructions: ~22 per (element, worker) + ~10 per element for the fused decode,
+# ~24 per element for the encode.
+DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 24.0
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
+NCU_TRAFFIC = {}
 
 
 def parse_args():
@@ -55,7 +61,7 @@ def parse_args():
     ap.add_argument("--no-kernels", action="store_true", help="skip the per-kernel isolated timings")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under a profiler: only warm-up + timed steps, no sampler, no extra legs")
-    ap.add_argument("--cpu-sample", type=int, default=1 << 23, help="elements per worker in the oracle sample")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 25, help="elements per worker in the oracle sample")
     a = ap.parse_args()
     if a.profile:
         a.no_cpu_baseline = a.no_e2e = a.no_kernels = True
@@ -161,20 +167,26 @@ class ClockSampler:
 class GpuState:
     """Device buffers of one replica: W gradients, W message buffers, side information, output."""
 
-    def __init__(self, dq, torch, cfg, dev):
+    def __init__(self, dq, torch, cfg, dev, share=None):
+        """share: another GpuState of the same workload whose gradients (and side information) are reused."""
         from dq_workloads.generators import DQSG
         self.dq, self.torch, self.cfg, self.dev = dq, torch, cfg, dev
         self.DQSG = DQSG
         self.params = [dq.binding.make_params(cfg.bucket, s.bits, s.levels, s.coarse_K, s.fine_M, s.alpha,
                                               s.dither_bits)
                        for s in cfg.workers]
-        self.grads_host = [torch.from_numpy(cfg.grad(w)).pin_memory() for w in range(cfg.W)]
-        self.grads = [g.to(dev, non_blocking=True) for g in self.grads_host]
+        if share is not None:
+            self.grads_host, self.grads = share.grads_host, share.grads
+        else:
+            self.grads_host = [torch.from_numpy(cfg.grad(w)).pin_memory() for w in range(cfg.W)]
+            self.grads = [g.to(dev, non_blocking=True) for g in self.grads_host]
         self.msg_buf = [dq.binding.alloc_message(cfg.n, p, dev) for p in self.params]
         self.msgs = [dq.Message(pk, sc, s.seed, w, s.kind, p)
                      for w, (s, p, (pk, sc)) in enumerate(zip(cfg.workers, self.params, self.msg_buf))]
         self.any_nested = any(s.kind != DQSG for s in cfg.workers)
-        if cfg.side_info is not None:
+        if cfg.side_info is not None and share is not None:
+            self.side_host, self.side = share.side_host, share.side
+        elif cfg.side_info is not None:
             self.side_host = torch.from_numpy(cfg.side_info()).pin_memory()
             self.side = self.side_host.to(dev)
         elif cfg.side_from_worker0:
@@ -254,7 +266,10 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
         by = encode_bytes(dq, n, s, cfg.bucket)
         name = f"encode_{'dqsg' if s.kind == st.DQSG else 'ndqsg'}_b{s.bits}"
         res[name] = {"ms": ms, "bytes": by, "gbs": by / ms / 1e6, "gelem_s": n / ms / 1e6,
-                     "frac_hbm": by / ms / 1e6 / hbm_peak, "rotating_buffers": rot}
+                     "frac_hbm": by / ms / 1e6 / hbm_peak, "rotating_buffers": rot,
+                     "alu_tinstr_s": ENC_INSTR_PER_ELEM * n / ms / 1e9,
+                     "frac_alu": ENC_INSTR_PER_ELEM * n / ms * 1e3 / alu_peak,
+                     "traffic": NCU_TRAFFIC.get(("encode", cfg.name, n, s.bits))}
     # decode: rotate over message sets / side / out copies so that nothing is L2-resident
     per_set = decode_bytes(dq, n, cfg.workers, cfg.bucket, st.any_nested)
     sets = max(2, min(6, -(-3 * L2_BYTES // per_set)))
@@ -271,10 +286,13 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
     launches = [(lambda a=msg_sets[i], b=sides[i], c=outs[i]: st.decode(a, b, c)) for i in range(sets)]
     ms = time_isolated(torch, launches, iters=12)
     elem_workers = n * cfg.W
+    alg_instr = DEC_INSTR_PER_ELEM_WORKER * elem_workers + DEC_INSTR_PER_ELEM * n
     res["decode_aggregate"] = {"ms": ms, "bytes": per_set, "gbs": per_set / ms / 1e6, "gelem_s": n / ms / 1e6,
                                "frac_hbm": per_set / ms / 1e6 / hbm_peak,
                                "gelem_worker_s": elem_workers / ms / 1e6, "rotating_buffers": sets,
-                               "alu_peak_lane_instr_s": alu_peak}
+                               "alu_tinstr_s": alg_instr / ms / 1e9, "frac_alu": alg_instr / ms * 1e3 / alu_peak,
+                               "alu_peak_tinstr_s": alu_peak / 1e12,
+                               "traffic": NCU_TRAFFIC.get(("decode", cfg.name, n))}
     return res
 
 
@@ -483,6 +501,25 @@ def main():
     value = whole_job_value(step_bytes, world, ms_per_step)
 
     kernels = {} if args.no_kernels else kernel_timings(st, hbm_peak, sm_max_mhz)
+    # the same workload with the 16-bit dither stream (half the generator work), timed beside the default
+    alt = None
+    if not args.no_kernels and args.dither_bits == 32:
+        import dq_workloads as wl
+        cfg16 = wl.with_dither_bits(make_workload(args, rank), 16)
+        st16 = GpuState(dq, torch, cfg16, dev, share=st)
+        for _ in range(3):
+            st16.step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            st16.step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms16 = max_over_ranks([e0.elapsed_time(e1) / args.steps], dev)[0]
+        alt = {"ms_per_step": ms16, "value": whole_job_value(step_bytes, world, ms16), "unit": "GB/s",
+               "kernels": kernel_timings(st16, hbm_peak, sm_max_mhz)}
+        del st16
     e2e = None
     if not args.no_e2e:
         dt, h2d, d2h, _ = run_e2e(st, max(1, min(args.steps, 3)))
@@ -493,19 +530,33 @@ def main():
     if rank == 0:
         n_enc = cfg.W
         enc_share = enc_ms / (enc_ms + dec_ms)
+        roofline_encode = None
         if kernels:
+            # the dominant kernel = the one with the largest share of the step's device time
             enc_names = [k for k in kernels if k.startswith("encode")]
-            dom = max(enc_names, key=lambda k: sum(1 for s in cfg.workers
-                                                   if k == f"encode_{'dqsg' if s.kind == 0 else 'ndqsg'}_b{s.bits}"))
-            kd = kernels[dom]
-            roofline = {"kernel": dom, "bound": "hbm", "achieved": kd["gbs"], "peak": hbm_peak, "unit": "GB/s",
-                        "frac": kd["gbs"] / hbm_peak, "traffic": None, "peak_source": f"of {peak_src}",
-                        "frac_of_nominal_8TBs": kd["gbs"] / HBM_NOMINAL_GBS}
+            count = {k: sum(1 for s in cfg.workers if k == f"encode_{'dqsg' if s.kind == 0 else 'ndqsg'}_b{s.bits}")
+                     for k in enc_names}
+            dom_enc = max(enc_names, key=lambda k: count[k] * kernels[k]["ms"])
+            ke, kd = kernels[dom_enc], kernels["decode_aggregate"]
+            roofline_encode = {"kernel": dom_enc, "bound": "hbm", "achieved": ke["gbs"], "peak": hbm_peak,
+                               "unit": "GB/s", "frac": ke["gbs"] / hbm_peak, "traffic": ke["traffic"],
+                               "peak_source": f"of {peak_src}", "frac_of_nominal_8TBs": ke["gbs"] / HBM_NOMINAL_GBS,
+                               "launches_per_step": count[dom_enc], "frac_alu": ke["frac_alu"]}
+            roofline_decode = {"kernel": "decode_aggregate", "bound": "alu", "achieved": kd["alu_tinstr_s"],
+                               "peak": kd["alu_peak_tinstr_s"], "unit": "Tlane-instr/s", "frac": kd["frac_alu"],
+                               "traffic": kd["traffic"],
+                               "peak_source": "148 SMs x 4 schedulers x 32 lanes x max SM clock",
+                               "hbm_gbs": kd["gbs"], "frac_hbm": kd["frac_hbm"], "launches_per_step": 1}
+            if kd["ms"] >= count[dom_enc] * ke["ms"]:
+                roofline = roofline_decode
+            else:
+                roofline, roofline_encode = roofline_encode, None
         else:
             avg_enc_ms = enc_ms / n_enc
             gbs = enc_bytes / n_enc / avg_enc_ms / 1e6
             roofline = {"kernel": "encode (in-step average)", "bound": "hbm", "achieved": gbs, "peak": hbm_peak,
                         "unit": "GB/s", "frac": gbs / hbm_peak, "traffic": None, "peak_source": f"of {peak_src}"}
+            roofline_decode = None
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -517,6 +568,12 @@ def main():
                        "encode_bytes": enc_bytes, "decode_bytes": dec_bytes},
             "roofline": roofline, "kernels": kernels, "clocks": clocks, "gpu_launches": launches,
         }
+        if roofline_encode is not None:
+            line["roofline_encode"] = roofline_encode
+        if roofline_decode is not None and roofline_decode is not roofline:
+            line["roofline_decode"] = roofline_decode
+        if alt is not None:
+            line["dither16"] = alt
         if e2e:
             line["e2e"] = e2e
         if not args.no_cpu_baseline:

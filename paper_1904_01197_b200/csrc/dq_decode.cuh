@@ -67,29 +67,23 @@ __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS
 }
 
 template <int BITS>
-__device__ __forceinline__ void load_row_words(const uint32_t* src, bool full_row, uint64_t first_word,
-                                               uint64_t num_words, uint32_t (&words)[BITS])
+__device__ __forceinline__ void load_row_words(const uint32_t* src, uint32_t (&words)[BITS])
 {
-    if (full_row) {
-        if constexpr (BITS % 4 == 0) {
+    if constexpr (BITS % 4 == 0) {
 #pragma unroll
-            for (int j = 0; j < BITS; j += 4) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(src) + (j >> 2));
-                words[j] = v.x; words[j + 1] = v.y; words[j + 2] = v.z; words[j + 3] = v.w;
-            }
-        } else if constexpr (BITS % 2 == 0) {
+        for (int j = 0; j < BITS; j += 4) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(src) + (j >> 2));
+            words[j] = v.x; words[j + 1] = v.y; words[j + 2] = v.z; words[j + 3] = v.w;
+        }
+    } else if constexpr (BITS % 2 == 0) {
 #pragma unroll
-            for (int j = 0; j < BITS; j += 2) {
-                const uint2 v = __ldg(reinterpret_cast<const uint2*>(src) + (j >> 1));
-                words[j] = v.x; words[j + 1] = v.y;
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < BITS; ++j) words[j] = __ldg(src + j);
+        for (int j = 0; j < BITS; j += 2) {
+            const uint2 v = __ldg(reinterpret_cast<const uint2*>(src) + (j >> 1));
+            words[j] = v.x; words[j + 1] = v.y;
         }
     } else {
 #pragma unroll
-        for (int j = 0; j < BITS; ++j) words[j] = (first_word + j < num_words) ? __ldg(src + j) : 0u;
+        for (int j = 0; j < BITS; ++j) words[j] = __ldg(src + j);
     }
 }
 
@@ -97,12 +91,12 @@ __device__ __forceinline__ void load_row_words(const uint32_t* src, bool full_ro
 //   DQSG:  g~ = (kappa/s) ((k - s) - delta); (k - s + 1.5) - f rounds once to the same value.
 //   NDQSG: r = (m - delta) - y a;  jj = rint(r / K);  q1^ = m - K jj;  g~ = beta (q1^ - delta) [+ (1-alpha^2) y]
 template <int BITS, uint32_t KIND, int DITH>
-__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
-                                           uint64_t n, const float* __restrict__ side_row, float (&acc)[32],
+__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket,
+                                           const float* __restrict__ side_row, float (&acc)[32],
                                            uint32_t* status)
 {
     uint32_t words[BITS];
-    load_row_words<BITS>(wk.packed + row * BITS, full_row, row * BITS, (n * BITS + 31u) >> 5, words);
+    load_row_words<BITS>(wk.packed + row * BITS, words);
 
     const float kappa = __ldg(wk.scale + bucket);
     if (status != nullptr && !(fabsf(kappa) <= 3.402823466e38f)) atomicOr(status, 0x1u);
@@ -126,14 +120,8 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
         for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (KIND != kDecDqsg) {
-                if (full_row) {
-                    const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + (PASS / 4) * h + q);
-                    y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        y[e] = (row * 32u + PASS * h + 4u * q + e < n) ? __ldg(side_row + PASS * h + 4 * q + e) : 0.0f;
-                }
+                const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + (PASS / 4) * h + q);
+                y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -170,19 +158,69 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
 }
 
 template <uint32_t KIND, int DITH>
-__device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket, bool full_row,
-                                                uint64_t n, const float* side_row, float (&acc)[32],
-                                                uint32_t* status)
+__device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket,
+                                                const float* side_row, float (&acc)[32], uint32_t* status)
 {
     switch (wk.bits) {
-        case 1: decode_row<1, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 2: decode_row<2, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 3: decode_row<3, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 4: decode_row<4, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 5: decode_row<5, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 6: decode_row<6, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        case 7: decode_row<7, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
-        default: decode_row<8, KIND, DITH>(wk, row, bucket, full_row, n, side_row, acc, status); break;
+        case 1: decode_row<1, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 2: decode_row<2, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 3: decode_row<3, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 4: decode_row<4, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 5: decode_row<5, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 6: decode_row<6, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 7: decode_row<7, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        default: decode_row<8, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+    }
+}
+
+// The last row of a gradient whose length is not a multiple of 32: one element at a time, everything at run
+// time.  Same arithmetic, in the same order, as decode_row.
+template <int DITH>
+__device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t row, uint64_t bucket, uint32_t nvalid)
+{
+    for (uint32_t e = 0; e < nvalid; ++e) {
+        const uint64_t i = row * 32u + e;
+        const float yy = args.side ? __ldg(args.side + i) : 0.0f;
+        float acc = 0.0f;
+        for (uint32_t w = 0; w < args.W; ++w) {
+            const DecWorker& wk = args.w[w];
+            const uint32_t bits = wk.bits;
+            const uint64_t bit = i * bits;
+            const uint64_t num_words = (args.n * bits + 31u) >> 5;
+            uint32_t lo = __ldg(wk.packed + (bit >> 5));
+            const uint32_t sh = (uint32_t)(bit & 31u);
+            uint32_t code = lo >> sh;
+            if (sh + bits > 32u && (bit >> 5) + 1u < num_words) code |= __ldg(wk.packed + (bit >> 5) + 1u) << (32u - sh);
+            code &= (1u << bits) - 1u;
+            uint32_t ctr[1], rnd[1][4];
+            float f;
+            if (DITH == 16) {
+                ctr[0] = (uint32_t)(i >> 3);
+                philox4x32_10_xN<1>(ctr, wk.ps, rnd);
+                f = dither16_f12(rnd[0][(i & 7u) >> 1], (int)(i & 1u));
+            } else {
+                ctr[0] = (uint32_t)(i >> 2);
+                philox4x32_10_xN<1>(ctr, wk.ps, rnd);
+                f = dither_f12(rnd[0][i & 3u]);
+            }
+            const float kappa = __ldg(wk.scale + bucket);
+            if (args.status != nullptr && !(fabsf(kappa) <= 3.402823466e38f)) atomicOr(args.status, 0x1u);
+            const float X = __fadd_rn(__uint_as_float((code << 1) | 0x4A800000u), -wk.cconst);
+            float gt;
+            if (wk.kind == kDecDqsg) {
+                gt = __fmul_rn(__fdiv_rn(kappa, wk.s), __fadd_rn(X, -f));
+            } else {
+                const float a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
+                const float c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);
+                const float r = __fmaf_rn(-yy, a, __fadd_rn(X, -f));
+                const float t = (wk.kind == kDecNdqsgAnyK) ? __fdiv_rn(r, wk.Kf) : __fmul_rn(r, wk.invK);
+                const float jj = __fadd_rn(__fadd_rn(t, kMagic), -kMagic);
+                const float d = __fadd_rn(__fmaf_rn(-wk.Kf, jj, X), -f);
+                gt = (wk.alpha == 1.0f) ? __fmul_rn(c, d) : __fmaf_rn(c, d, __fmul_rn(wk.one_m_alpha2, yy));
+            }
+            acc = __fadd_rn(acc, gt);
+        }
+        args.out[i] = (args.invW != 0.0f) ? __fmul_rn(acc, args.invW) : __fdiv_rn(acc, args.Wf);
     }
 }
 
@@ -199,9 +237,11 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     const uint64_t row = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= args.rows) return;
     const uint64_t base = row * 32u;
-    const bool full_row = (base + 32u <= args.n);
-    const uint32_t nvalid = full_row ? 32u : (uint32_t)(args.n - base);
     const uint64_t bucket = row / args.rows_per_bucket;
+    if (base + 32u > args.n) {
+        decode_partial_row<DITH>(args, row, bucket, (uint32_t)(args.n - base));
+        return;
+    }
     const float* side_row = args.side ? args.side + base : nullptr;
 
     float acc[32];
@@ -211,10 +251,10 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     for (uint32_t w = 0; w < args.W; ++w) {
         const DecWorker& wk = args.w[w];
         switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
-            default: decode_row_bits<kDecNdqsgAnyK, DITH>(wk, row, bucket, full_row, args.n, side_row, acc, args.status); break;
+            case kDecDqsg: decode_row_bits<kDecDqsg, DITH>(wk, row, bucket, side_row, acc, args.status); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH>(wk, row, bucket, side_row, acc, args.status); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH>(wk, row, bucket, side_row, acc, args.status); break;
+            default: decode_row_bits<kDecNdqsgAnyK, DITH>(wk, row, bucket, side_row, acc, args.status); break;
         }
     }
 
@@ -222,16 +262,10 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     for (int e = 0; e < 32; ++e)
         acc[e] = (args.invW != 0.0f) ? __fmul_rn(acc[e], args.invW) : __fdiv_rn(acc[e], args.Wf);
 
-    if (full_row) {
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-            reinterpret_cast<float4*>(args.out + base)[c] =
-                make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
-    } else {
-#pragma unroll
-        for (int e = 0; e < 32; ++e)
-            if ((uint32_t)e < nvalid) args.out[base + e] = acc[e];
-    }
+    for (int c = 0; c < 8; ++c)
+        reinterpret_cast<float4*>(args.out + base)[c] =
+            make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
 }
 
 }  // namespace dq
