@@ -41,7 +41,11 @@ SM_COUNT, ISSUE_PER_SM_CLK, LANES = 148, 4, 32           # ALU-issue ceiling: SM
 DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 24.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_075_904,    # profiles/encode_kernel_ndqsg_resnet50.md
+    ("encode", "ndqsg_resnet50", 25_557_032, 3): 106_433_024,
+    ("decode", "ndqsg_resnet50", 25_557_032): 220_729_088,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
+}
 
 
 def parse_args():
@@ -269,7 +273,7 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
                      "frac_hbm": by / ms / 1e6 / hbm_peak, "rotating_buffers": rot,
                      "alu_tinstr_s": ENC_INSTR_PER_ELEM * n / ms / 1e9,
                      "frac_alu": ENC_INSTR_PER_ELEM * n / ms * 1e3 / alu_peak,
-                     "traffic": NCU_TRAFFIC.get(("encode", cfg.name, n, s.bits))}
+                     "traffic": NCU_TRAFFIC.get(("encode", cfg.name, n, s.bits)) if s.dither_bits == 32 else None}
     # decode: rotate over message sets / side / out copies so that nothing is L2-resident
     per_set = decode_bytes(dq, n, cfg.workers, cfg.bucket, st.any_nested)
     sets = max(2, min(6, -(-3 * L2_BYTES // per_set)))
@@ -292,7 +296,8 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
                                "gelem_worker_s": elem_workers / ms / 1e6, "rotating_buffers": sets,
                                "alu_tinstr_s": alg_instr / ms / 1e9, "frac_alu": alg_instr / ms * 1e3 / alu_peak,
                                "alu_peak_tinstr_s": alu_peak / 1e12,
-                               "traffic": NCU_TRAFFIC.get(("decode", cfg.name, n))}
+                               "traffic": (NCU_TRAFFIC.get(("decode", cfg.name, n))
+                                           if cfg.workers[0].dither_bits == 32 else None)}
     return res
 
 

@@ -95,8 +95,10 @@ __device__ __forceinline__ float dither_f12(uint32_t x)
 // 16-bit stream: half-word h -> f = 1 + (2h+1) 2^-17 in [1, 2); the dither is again f - 1.5 (exact).
 __device__ __forceinline__ float dither16_f12(uint32_t word, int high)
 {
-    const uint32_t v = high ? (word >> 9) : (word << 7);
-    return __uint_as_float((v & 0x007FFF80u) | 0x3F800040u);
+    // h * 128 + 0x3F800040: the half-word lands in mantissa bits 7..22 and bit 6 makes the grid odd; the two
+    // fields do not overlap, so the multiply-add is the same as shift-and-or but needs a single constant.
+    const uint32_t h = high ? (word >> 16) : (word & 0xFFFFu);
+    return __uint_as_float(h * 128u + 0x3F800040u);
 }
 
 // f of element t (0 .. 4*EPB-1) of a group of four Philox blocks; EPB = elements per block (4 or 8).
