@@ -93,6 +93,9 @@ def lib():
         L.dqo_decode_aggregate.argtypes = [C.POINTER(_Msg), C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64,
                                            f32p, f32p, f32p, i32p, C.c_int]
         L.dqo_decode_aggregate.restype = C.c_int
+        L.dqo_decode_aggregate_running.argtypes = [C.POINTER(_Msg), C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64,
+                                                   f32p, f32p, i32p, C.c_int]
+        L.dqo_decode_aggregate_running.restype = C.c_int
         L.dqo_nearest_coset_bruteforce.argtypes = [C.c_uint32, C.c_int32, C.c_double, C.c_double,
                                                    C.c_double, C.c_int32, C.POINTER(C.c_double)]
         L.dqo_nearest_coset_bruteforce.restype = C.c_int32
@@ -237,8 +240,10 @@ class Msg:
 
 
 def decode_aggregate(msgs: Sequence[Msg], n: int, step: int, side_info: Optional[np.ndarray] = None,
-                     i0: int = 0, want_recon: bool = False, want_qhat: bool = False, threads: int = 1):
-    """Returns out_avg fp32[n] (plus recon fp32[W][n] and/or qhat int32[W][n] when asked)."""
+                     i0: int = 0, want_recon: bool = False, want_qhat: bool = False, threads: int = 1,
+                     running: bool = False):
+    """Returns out_avg fp32[n] (plus recon fp32[W][n] and/or qhat int32[W][n] when asked).
+    running=True: Algorithm 2's server loop, side information = mean of everything decoded before."""
     W = len(msgs)
     arr = (_Msg * max(1, W))()
     for w, m in enumerate(msgs):
@@ -250,9 +255,14 @@ def decode_aggregate(msgs: Sequence[Msg], n: int, step: int, side_info: Optional
     out = np.zeros(max(1, n), dtype=np.float32)
     recon = np.zeros((max(1, W), max(1, n)), dtype=np.float32) if want_recon else None
     qhat = np.zeros((max(1, W), max(1, n)), dtype=np.int32) if want_qhat else None
-    _check(lib().dqo_decode_aggregate(arr, W, n, i0, step, _p(side_info, C.c_float), _p(out, C.c_float),
-                                      _p(recon, C.c_float), _p(qhat, C.c_int32), threads),
-           "decode_aggregate")
+    if running:
+        _check(lib().dqo_decode_aggregate_running(arr, W, n, i0, step, _p(out, C.c_float),
+                                                  _p(recon, C.c_float), _p(qhat, C.c_int32), threads),
+               "decode_aggregate_running")
+    else:
+        _check(lib().dqo_decode_aggregate(arr, W, n, i0, step, _p(side_info, C.c_float), _p(out, C.c_float),
+                                          _p(recon, C.c_float), _p(qhat, C.c_int32), threads),
+               "decode_aggregate")
     res = [out[:n]]
     if want_recon:
         res.append(recon[:, :n])

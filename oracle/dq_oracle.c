@@ -364,9 +364,9 @@ static float ndqsg_reconstruct(uint32_t m, int32_t K, float a, float beta, float
  * [W][n]) the resolved fine index of NDQSG workers (k - s is not stored for DQSG;
  * those rows get the code k).
  * ---------------------------------------------------------------------- */
-int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i0, uint64_t step,
-                         const float *side_info, float *out_avg,
-                         float *recon, int32_t *qhat, int threads)
+static int decode_aggregate_impl(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i0, uint64_t step,
+                                 const float *side_info, int running, float *out_avg,
+                                 float *recon, int32_t *qhat, int threads)
 {
     if (W == 0u) return DQO_BAD_ARG;
     for (uint32_t w = 0; w < W; ++w) {
@@ -381,7 +381,7 @@ int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i
         } else if (m->kind == DQO_KIND_NDQSG) {
             if (m->coarse_K < 2u || m->coarse_K > (1u << m->bits)) return DQO_BAD_ARG;
             if (!(m->fine_M > 0.0f) || !(m->alpha > 0.0f) || m->alpha > 1.0f) return DQO_BAD_ARG;
-            if (!side_info) return DQO_BAD_ARG;
+            if (running ? (w == 0u) : (side_info == NULL)) return DQO_BAD_ARG;
         } else {
             return DQO_BAD_ARG;
         }
@@ -409,8 +409,9 @@ int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i
                 float a = bucket_gain(A, kappa);
                 float beta = (m->alpha * kappa) / m->fine_M;
                 int32_t qh;
-                gt = ndqsg_reconstruct(code, (int32_t)m->coarse_K, a, beta, m->alpha, delta,
-                                       side_info[i], &qh);
+                /* Algorithm 2 as written: the side information is the mean of everything decoded so far */
+                float y = running ? acc * (1.0f / (float)w) : side_info[i];
+                gt = ndqsg_reconstruct(code, (int32_t)m->coarse_K, a, beta, m->alpha, delta, y, &qh);
                 if (qhat) qhat[(uint64_t)w * n + (uint64_t)i] = qh;
             }
             if (recon) recon[(uint64_t)w * n + (uint64_t)i] = gt;
@@ -419,6 +420,24 @@ int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i
         out_avg[i] = acc / (float)W;
     }
     return DQO_OK;
+}
+
+int dqo_decode_aggregate(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i0, uint64_t step,
+                         const float *side_info, float *out_avg,
+                         float *recon, int32_t *qhat, int threads)
+{
+    return decode_aggregate_impl(msgs, W, n, i0, step, side_info, 0, out_avg, recon, qhat, threads);
+}
+
+/* Algorithm 2, server loop, as written: the workers are visited in array order; a DQSG message (group P1) is
+ * reconstructed directly; an NDQSG message (group P2) is decoded against g_bar = the mean of all reconstructions
+ * before it, and g_bar is then updated with the new reconstruction.  With S the running fp32 sum and w the number
+ * of workers already decoded, g_bar = S * (1/w) (reciprocal rounded once).  The first message must be DQSG.
+ * The result is the mean over all W. */
+int dqo_decode_aggregate_running(const dqo_msg *msgs, uint32_t W, uint64_t n, uint64_t i0, uint64_t step,
+                                 float *out_avg, float *recon, int32_t *qhat, int threads)
+{
+    return decode_aggregate_impl(msgs, W, n, i0, step, NULL, 1, out_avg, recon, qhat, threads);
 }
 
 /* ------------------------------------------------------------------------
