@@ -289,6 +289,16 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
         outs.append(torch.empty_like(st.out))
     launches = [(lambda a=msg_sets[i], b=sides[i], c=outs[i]: st.decode(a, b, c)) for i in range(sets)]
     ms = time_isolated(torch, launches, iters=12)
+    if st.any_nested and cfg.workers[0].kind == st.DQSG:
+        # Algorithm 2's own server loop on the same messages: side information = running mean, no vector read
+        run_l = [(lambda a=msg_sets[i], c=outs[i]: dq.ndqsg_decode_aggregate_running(a, n, cfg.step, c))
+                 for i in range(sets)]
+        ms_run = time_isolated(torch, run_l, iters=12)
+        by_run = per_set - 4 * n
+        res["decode_aggregate_running_mean"] = {"ms": ms_run, "bytes": by_run, "gbs": by_run / ms_run / 1e6,
+                                                "gelem_s": n / ms_run / 1e6,
+                                                "frac_hbm": by_run / ms_run / 1e6 / hbm_peak,
+                                                "gelem_worker_s": n * cfg.W / ms_run / 1e6}
     elem_workers = n * cfg.W
     alg_instr = DEC_INSTR_PER_ELEM_WORKER * elem_workers + DEC_INSTR_PER_ELEM * n
     res["decode_aggregate"] = {"ms": ms, "bytes": per_set, "gbs": per_set / ms / 1e6, "gelem_s": n / ms / 1e6,

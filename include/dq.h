@@ -132,6 +132,17 @@ dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uin
                                  void* cuda_stream);
 
 /*
+ * ndqsg_decode_aggregate_running -- the server loop of Algorithm 2 as written: the messages are visited in
+ * array order; a DQSG message (group P1) is reconstructed directly; an NDQSG message (group P2) is resolved
+ * against g_bar = the mean of all reconstructions before it, which is then updated with the new one ("update
+ * g_bar using g_p").  g_bar is S * (1/w) with S the running fp32 sum and w the number of messages already
+ * decoded, so no side-information vector is read.  msgs[0] must be a DQSG message.  The mean of all W
+ * reconstructions is written.  Other arguments as for ndqsg_decode_aggregate.
+ */
+dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                         float* out_avg, uint32_t* status_word, void* cuda_stream);
+
+/*
  * Host-buffer variants.  Every data pointer (grad, out_packed, out_scale, the packed/scale pointers
  * inside msgs, side_info, out_avg) is HOST memory (pinned memory makes the copies asynchronous);
  * `workspace` is device memory of at least the stated size, 256-byte aligned, provided by the caller.

@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     ndqsg_encode,
     dqsg_decode_aggregate,
     ndqsg_decode_aggregate,
+    ndqsg_decode_aggregate_running,
     encode_workspace_bytes,
     decode_workspace_bytes,
     dqsg_encode_host,

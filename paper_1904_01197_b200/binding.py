@@ -62,6 +62,8 @@ def lib() -> C.CDLL:
         L.dqsg_decode_aggregate.restype = C.c_int
         L.ndqsg_decode_aggregate.argtypes = [pm, u32, u64, u64, vp, vp, vp, vp]
         L.ndqsg_decode_aggregate.restype = C.c_int
+        L.ndqsg_decode_aggregate_running.argtypes = [pm, u32, u64, u64, vp, vp, vp]
+        L.ndqsg_decode_aggregate_running.restype = C.c_int
         L.dq_encode_workspace_bytes.argtypes = [u64, pp]; L.dq_encode_workspace_bytes.restype = u64
         L.dq_decode_workspace_bytes.argtypes = [pm, u32, u64, C.c_int]; L.dq_decode_workspace_bytes.restype = u64
         for f in (L.dqsg_encode_host, L.ndqsg_encode_host):
@@ -202,6 +204,19 @@ def ndqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, side_info
                                         _dev_ptr(out_avg, torch.float32, "out_avg"),
                                         _dev_ptr(status_word, torch.int32, "status_word"), _stream_ptr(stream)),
            "ndqsg_decode_aggregate")
+    return out_avg
+
+
+def ndqsg_decode_aggregate_running(msgs: Sequence[Message], n: int, step: int,
+                                   out_avg: Optional[torch.Tensor] = None,
+                                   status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Algorithm 2's server loop: NDQSG messages are decoded against the mean of the messages before them."""
+    if out_avg is None:
+        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+    _check(lib().ndqsg_decode_aggregate_running(_msg_array(msgs), len(msgs), n, step,
+                                                _dev_ptr(out_avg, torch.float32, "out_avg"),
+                                                _dev_ptr(status_word, torch.int32, "status_word"),
+                                                _stream_ptr(stream)), "ndqsg_decode_aggregate_running")
     return out_avg
 
 

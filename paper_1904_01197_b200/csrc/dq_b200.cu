@@ -231,7 +231,8 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
 }
 
 dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, const float* side_info,
-                        float* out_avg, uint32_t* status_word, bool allow_nested, cudaStream_t st)
+                        float* out_avg, uint32_t* status_word, bool allow_nested, cudaStream_t st,
+                        bool running = false)
 {
     if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
     static thread_local dq::DecodeArgs a;    // ~10 KB: keep it off the stack
@@ -267,18 +268,22 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
             d.one_m_alpha2 = 1.0f - a2;
             d.Kf = (float)m.p.coarse_K;
             d.invK = 1.0f / d.Kf;
+            if (running) {
+                if (w == 0u) return DQ_ERR_INVALID_ARG;      // nothing decoded yet to serve as side information
+                d.rcp_count = 1.0f / (float)w;
+            }
         }
     }
     if (n == 0) return DQ_OK;
     if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
     if (!out_avg) return DQ_ERR_INVALID_ARG;
-    if (any_nested && !side_info) return DQ_ERR_INVALID_ARG;
+    if (any_nested && !running && !side_info) return DQ_ERR_INVALID_ARG;
     if (!aligned16(out_avg) || (side_info && !aligned16(side_info))) return DQ_ERR_ALIGNMENT;
     for (uint32_t w = 0; w < W; ++w) {
         if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
         if (!aligned16(msgs[w].packed) || !aligned16(msgs[w].scale)) return DQ_ERR_ALIGNMENT;
     }
-    a.side = any_nested ? side_info : nullptr;
+    a.side = (any_nested && !running) ? side_info : nullptr;
     a.out = out_avg;
     a.status = status_word;
     a.n = n;
@@ -289,8 +294,15 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
     const uint64_t grid64 = (a.rows + dq::kDecThreads - 1u) / dq::kDecThreads;
     if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
-    if (msgs[0].p.dither_bits == 16u) dq::decode_aggregate_kernel<16><<<(uint32_t)grid64, dq::kDecThreads, 0, st>>>(a);
-    else dq::decode_aggregate_kernel<32><<<(uint32_t)grid64, dq::kDecThreads, 0, st>>>(a);
+    const bool d16 = (msgs[0].p.dither_bits == 16u);
+    const uint32_t grid = (uint32_t)grid64;
+    if (running && any_nested) {
+        if (d16) dq::decode_aggregate_kernel<16, true><<<grid, dq::kDecThreads, 0, st>>>(a);
+        else dq::decode_aggregate_kernel<32, true><<<grid, dq::kDecThreads, 0, st>>>(a);
+    } else {
+        if (d16) dq::decode_aggregate_kernel<16, false><<<grid, dq::kDecThreads, 0, st>>>(a);
+        else dq::decode_aggregate_kernel<32, false><<<grid, dq::kDecThreads, 0, st>>>(a);
+    }
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;
@@ -344,6 +356,13 @@ dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uin
 {
     return decode_common(msgs, W, n, step, side_info, out_avg, status_word, true,
                          static_cast<cudaStream_t>(cuda_stream));
+}
+
+dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, float* out_avg,
+                                         uint32_t* status_word, void* cuda_stream)
+{
+    return decode_common(msgs, W, n, step, nullptr, out_avg, status_word, true,
+                         static_cast<cudaStream_t>(cuda_stream), true);
 }
 
 // ------------------------------------------------------------------------------------------------ host buffers

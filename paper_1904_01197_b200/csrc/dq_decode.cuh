@@ -32,6 +32,7 @@ struct DecWorker {
     float one_m_alpha2;   // 1 - alpha*alpha
     float Kf;             // (float)K
     float invK;           // 1/K (exact when K is a power of two)
+    float rcp_count;      // running-mean mode: 1 / (number of workers before this one)
 };
 
 struct DecodeArgs {
@@ -90,7 +91,7 @@ __device__ __forceinline__ void load_row_words(const uint32_t* src, uint32_t (&w
 // One worker's contribution to the 32 accumulators of a row.
 //   DQSG:  g~ = (kappa/s) ((k - s) - delta); (k - s + 1.5) - f rounds once to the same value.
 //   NDQSG: r = (m - delta) - y a;  jj = rint(r / K);  q1^ = m - K jj;  g~ = beta (q1^ - delta) [+ (1-alpha^2) y]
-template <int BITS, uint32_t KIND, int DITH>
+template <int BITS, uint32_t KIND, int DITH, bool RUN>
 __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket,
                                            const float* __restrict__ side_row, float (&acc)[32],
                                            uint32_t* status)
@@ -119,7 +120,7 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
 #pragma unroll
         for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-            if (KIND != kDecDqsg) {
+            if (KIND != kDecDqsg && !RUN) {
                 const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + (PASS / 4) * h + q);
                 y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
             }
@@ -134,7 +135,9 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
                     const float d = __fadd_rn(X, -f);                      // (k - s) - delta
                     gt = __fmul_rn(c, d);
                 } else {
-                    const float yy = y[e];
+                    // side information: the given vector, or (Algorithm 2 as written) the mean of the
+                    // reconstructions accumulated so far
+                    const float yy = RUN ? __fmul_rn(acc[idx], wk.rcp_count) : y[e];
                     const float r1 = __fadd_rn(X, -f);                     // m - delta
                     const float r = __fmaf_rn(-yy, a, r1);
                     float jj;
@@ -157,30 +160,30 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
     }
 }
 
-template <uint32_t KIND, int DITH>
+template <uint32_t KIND, int DITH, bool RUN>
 __device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket,
                                                 const float* side_row, float (&acc)[32], uint32_t* status)
 {
     switch (wk.bits) {
-        case 1: decode_row<1, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        case 2: decode_row<2, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        case 3: decode_row<3, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        case 4: decode_row<4, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        case 5: decode_row<5, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        case 6: decode_row<6, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        case 7: decode_row<7, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
-        default: decode_row<8, KIND, DITH>(wk, row, bucket, side_row, acc, status); break;
+        case 1: decode_row<1, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 2: decode_row<2, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 3: decode_row<3, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 4: decode_row<4, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 5: decode_row<5, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 6: decode_row<6, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 7: decode_row<7, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        default: decode_row<8, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
     }
 }
 
 // The last row of a gradient whose length is not a multiple of 32: one element at a time, everything at run
 // time.  Same arithmetic, in the same order, as decode_row.
-template <int DITH>
+template <int DITH, bool RUN>
 __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t row, uint64_t bucket, uint32_t nvalid)
 {
     for (uint32_t e = 0; e < nvalid; ++e) {
         const uint64_t i = row * 32u + e;
-        const float yy = args.side ? __ldg(args.side + i) : 0.0f;
+        const float yside = (!RUN && args.side) ? __ldg(args.side + i) : 0.0f;
         float acc = 0.0f;
         for (uint32_t w = 0; w < args.W; ++w) {
             const DecWorker& wk = args.w[w];
@@ -210,6 +213,7 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t
             if (wk.kind == kDecDqsg) {
                 gt = __fmul_rn(__fdiv_rn(kappa, wk.s), __fadd_rn(X, -f));
             } else {
+                const float yy = RUN ? __fmul_rn(acc, wk.rcp_count) : yside;
                 const float a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
                 const float c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);
                 const float r = __fmaf_rn(-yy, a, __fadd_rn(X, -f));
@@ -230,7 +234,7 @@ constexpr int kDecThreads = 128;
 #endif
 constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;
 
-template <int DITH>
+template <int DITH, bool RUN>
 __global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
 decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
 {
@@ -239,7 +243,7 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     const uint64_t base = row * 32u;
     const uint64_t bucket = row / args.rows_per_bucket;
     if (base + 32u > args.n) {
-        decode_partial_row<DITH>(args, row, bucket, (uint32_t)(args.n - base));
+        decode_partial_row<DITH, RUN>(args, row, bucket, (uint32_t)(args.n - base));
         return;
     }
     const float* side_row = args.side ? args.side + base : nullptr;
@@ -251,10 +255,10 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     for (uint32_t w = 0; w < args.W; ++w) {
         const DecWorker& wk = args.w[w];
         switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg, DITH>(wk, row, bucket, side_row, acc, args.status); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH>(wk, row, bucket, side_row, acc, args.status); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH>(wk, row, bucket, side_row, acc, args.status); break;
-            default: decode_row_bits<kDecNdqsgAnyK, DITH>(wk, row, bucket, side_row, acc, args.status); break;
+            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
+            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
         }
     }
 
