@@ -18,8 +18,10 @@ from typing import List, Optional, Sequence
 import numpy as np
 
 _HERE = Path(__file__).resolve().parent
-_SRC = _HERE / "dq_oracle.c"
-_OUT = _HERE / "_build" / "libdq_oracle.so"
+# DQ_ORACLE_SOURCE / DQ_ORACLE_LIBRARY let the mutation test point a subprocess at a deliberately broken copy of
+# the C file (to check that the pins notice); nothing else sets them.
+_SRC = Path(os.environ.get("DQ_ORACLE_SOURCE", _HERE / "dq_oracle.c"))
+_OUT = Path(os.environ.get("DQ_ORACLE_LIBRARY", _HERE / "_build" / "libdq_oracle.so"))
 
 KIND_DQSG = 0
 KIND_NDQSG = 1
