@@ -290,6 +290,7 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.rows = (n + 31u) / 32u;
     a.W = W;
     a.rows_per_bucket = msgs[0].p.bucket / 32u;
+    a.half_bias_bits = 0x4A800000u;
     a.Wf = (float)W;
     a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
     const uint64_t grid64 = (a.rows + dq::kDecThreads - 1u) / dq::kDecThreads;

@@ -43,6 +43,7 @@ struct DecodeArgs {
     uint64_t rows;            // ceil(n / 32)
     uint32_t W;
     uint32_t rows_per_bucket; // B / 32
+    uint32_t half_bias_bits;  // 0x4A800000 (bit pattern of 2^22), passed in so that it lives in a register
     float Wf;
     float invW;               // 1/W when W is a power of two, else 0
     DecWorker w[64];
@@ -52,7 +53,7 @@ struct DecodeArgs {
 // 2^22 with the code in mantissa bits 1.., i.e. the value 2^22 + code (floats in [2^22, 2^23) step by 1/2).
 // Subtracting a constant then gives code - c exactly.
 template <int BITS>
-__device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS], int idx)
+__device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS], int idx, uint32_t bias_bits)
 {
     const int bit = idx * BITS;
     const int wi = bit >> 5;
@@ -64,7 +65,7 @@ __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS
     } else {
         v = __funnelshift_r(words[wi], words[(wi + 1) % BITS], sh - 1);
     }
-    return __uint_as_float((v & mask2) | 0x4A800000u);
+    return __uint_as_float((v & mask2) | bias_bits);          // one logic op: (v & immediate) | register
 }
 
 template <int BITS>
@@ -94,7 +95,7 @@ __device__ __forceinline__ void load_row_words(const uint32_t* src, uint32_t (&w
 template <int BITS, uint32_t KIND, int DITH, bool RUN>
 __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket,
                                            const float* __restrict__ side_row, float (&acc)[32],
-                                           uint32_t* status)
+                                           uint32_t* status, uint32_t bias_bits)
 {
     uint32_t words[BITS];
     load_row_words<BITS>(wk.packed + row * BITS, words);
@@ -129,7 +130,7 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
                 const int t = 4 * q + e;
                 const int idx = PASS * h + t;
                 const float f = dither_of<DITH>(rnd, t);
-                const float X = __fadd_rn(unpack_half_biased<BITS>(words, idx), -wk.cconst);
+                const float X = __fadd_rn(unpack_half_biased<BITS>(words, idx, bias_bits), -wk.cconst);
                 float gt;
                 if (KIND == kDecDqsg) {
                     const float d = __fadd_rn(X, -f);                      // (k - s) - delta
@@ -162,17 +163,18 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
 
 template <uint32_t KIND, int DITH, bool RUN>
 __device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket,
-                                                const float* side_row, float (&acc)[32], uint32_t* status)
+                                                const float* side_row, float (&acc)[32], uint32_t* status,
+                                                uint32_t bias_bits)
 {
     switch (wk.bits) {
-        case 1: decode_row<1, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        case 2: decode_row<2, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        case 3: decode_row<3, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        case 4: decode_row<4, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        case 5: decode_row<5, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        case 6: decode_row<6, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        case 7: decode_row<7, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
-        default: decode_row<8, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status); break;
+        case 1: decode_row<1, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 2: decode_row<2, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 3: decode_row<3, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 4: decode_row<4, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 5: decode_row<5, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 6: decode_row<6, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 7: decode_row<7, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        default: decode_row<8, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
     }
 }
 
@@ -255,10 +257,10 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     for (uint32_t w = 0; w < args.W; ++w) {
         const DecWorker& wk = args.w[w];
         switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
-            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, bucket, side_row, acc, args.status); break;
+            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
+            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
         }
     }
 

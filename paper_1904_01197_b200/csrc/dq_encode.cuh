@@ -314,8 +314,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         float mx = 0.0f;
 #pragma unroll
         for (int e = 0; e < 32; e += 2) mx = max3_abs(mx, x[e], x[e + 1]);
-        for (uint32_t off = args.lanes_per_bucket >> 1; off > 0; off >>= 1)
-            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+#pragma unroll
+        for (uint32_t off = 16; off > 0; off >>= 1) {
+            const float o = __shfl_xor_sync(0xFFFFFFFFu, mx, off);
+            if (off < args.lanes_per_bucket) mx = fmaxf(mx, o);
+        }
         __syncwarp();
         if (lane == 0) {
             const uint64_t next = tile + (uint64_t)kEncStages * stride;
@@ -325,21 +328,25 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                               (int32_t)(next * kTileRows + warp * 32u));
             }
         }
-        const uint64_t row = tile * kTileRows + warp * 32u + lane;       // row index in the gradient
+        const uint32_t row = (uint32_t)tile * kTileRows + warp * 32u + lane;   // row index in the gradient (< 2^29)
         if (wpb > 1u) {
             if (lane == 0) warp_max[k & 1u][warp] = mx;
             named_bar_sync(1u + group, wpb * 32u);
-            mx = warp_max[k & 1u][group * wpb];
-            for (uint32_t i = 1; i < wpb; ++i) mx = fmaxf(mx, warp_max[k & 1u][group * wpb + i]);
-            if (lane == 0 && (warp % wpb) == 0u) args.scale[(row * 32u) >> args.bucket_log2] = mx;
+            // the maximum over the bucket's warps: all eight slots are read, the ones of other buckets ignored
+#pragma unroll
+            for (uint32_t i = 0; i < (uint32_t)kConsumerWarps; ++i) {
+                const float o = warp_max[k & 1u][i];
+                if (i / wpb == group) mx = fmaxf(mx, o);
+            }
+            if (lane == 0 && (warp % wpb) == 0u) args.scale[row >> (args.bucket_log2 - 5u)] = mx;
         } else if ((lane & (args.lanes_per_bucket - 1u)) == 0u) {
-            args.scale[(row * 32u) >> args.bucket_log2] = mx;
+            args.scale[row >> (args.bucket_log2 - 5u)] = mx;
         }
         const float a = bucket_gain(args.gain_num, mx);
 
         uint32_t out[BITS];
-        encode_row<BITS, MODE, DITH>(x, (uint32_t)row, a, args, out);
-        store_row_words<BITS>(args.packed + row * BITS, out);
+        encode_row<BITS, MODE, DITH>(x, row, a, args, out);
+        store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
     }
 }
 
