@@ -68,39 +68,29 @@ __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS
     return __uint_as_float((v & mask2) | bias_bits);          // one logic op: (v & immediate) | register
 }
 
-template <int BITS>
-__device__ __forceinline__ void load_row_words(const uint32_t* src, uint32_t (&words)[BITS])
+// A worker's packed words of one row (bits words, at most 8) and its bucket scale.
+__device__ __forceinline__ void load_worker_row(const DecWorker& wk, uint64_t row, uint64_t bucket,
+                                                uint32_t (&words)[8], float& kappa)
 {
-    if constexpr (BITS % 4 == 0) {
+    const uint32_t* src = wk.packed + row * wk.bits;
 #pragma unroll
-        for (int j = 0; j < BITS; j += 4) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(src) + (j >> 2));
-            words[j] = v.x; words[j + 1] = v.y; words[j + 2] = v.z; words[j + 3] = v.w;
-        }
-    } else if constexpr (BITS % 2 == 0) {
-#pragma unroll
-        for (int j = 0; j < BITS; j += 2) {
-            const uint2 v = __ldg(reinterpret_cast<const uint2*>(src) + (j >> 1));
-            words[j] = v.x; words[j + 1] = v.y;
-        }
-    } else {
-#pragma unroll
-        for (int j = 0; j < BITS; ++j) words[j] = __ldg(src + j);
-    }
+    for (uint32_t j = 0; j < 8; ++j)
+        if (j < wk.bits) words[j] = __ldg(src + j);
+    kappa = __ldg(wk.scale + bucket);
 }
 
 // One worker's contribution to the 32 accumulators of a row.
 //   DQSG:  g~ = (kappa/s) ((k - s) - delta); (k - s + 1.5) - f rounds once to the same value.
 //   NDQSG: r = (m - delta) - y a;  jj = rint(r / K);  q1^ = m - K jj;  g~ = beta (q1^ - delta) [+ (1-alpha^2) y]
 template <int BITS, uint32_t KIND, int DITH, bool RUN>
-__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, uint64_t bucket,
-                                           const float* __restrict__ side_row, float (&acc)[32],
+__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, const uint32_t (&cur)[8],
+                                           float kappa, const float* side_row, float (&acc)[32],
                                            uint32_t* status, uint32_t bias_bits)
 {
     uint32_t words[BITS];
-    load_row_words<BITS>(wk.packed + row * BITS, words);
+#pragma unroll
+    for (int j = 0; j < BITS; ++j) words[j] = cur[j];
 
-    const float kappa = __ldg(wk.scale + bucket);
     if (status != nullptr && !(fabsf(kappa) <= 3.402823466e38f)) atomicOr(status, 0x1u);
 
     float c, a = 0.0f;
@@ -122,7 +112,9 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
         for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (KIND != kDecDqsg && !RUN) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(side_row) + (PASS / 4) * h + q);
+                // the row's side information sits in shared memory, 16-byte pieces swizzled by (row & 7)
+                const uint32_t piece = (uint32_t)((PASS / 4) * h + q) ^ (threadIdx.x & 7u);
+                const float4 v = *reinterpret_cast<const float4*>(side_row + 4u * piece);
                 y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
             }
 #pragma unroll
@@ -162,19 +154,19 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, ui
 }
 
 template <uint32_t KIND, int DITH, bool RUN>
-__device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, uint64_t bucket,
-                                                const float* side_row, float (&acc)[32], uint32_t* status,
-                                                uint32_t bias_bits)
+__device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, const uint32_t (&cur)[8],
+                                                float kappa, const float* side_row, float (&acc)[32],
+                                                uint32_t* status, uint32_t bias_bits)
 {
     switch (wk.bits) {
-        case 1: decode_row<1, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        case 2: decode_row<2, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        case 3: decode_row<3, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        case 4: decode_row<4, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        case 5: decode_row<5, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        case 6: decode_row<6, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        case 7: decode_row<7, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
-        default: decode_row<8, KIND, DITH, RUN>(wk, row, bucket, side_row, acc, status, bias_bits); break;
+        case 1: decode_row<1, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        case 2: decode_row<2, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        case 3: decode_row<3, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        case 4: decode_row<4, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        case 5: decode_row<5, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        case 6: decode_row<6, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        case 7: decode_row<7, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+        default: decode_row<8, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
     }
 }
 
@@ -240,7 +232,26 @@ template <int DITH, bool RUN>
 __global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
 decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
 {
-    const uint64_t row = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // Side information of the CTA's 128 rows -> shared memory (coalesced loads, 16-byte pieces swizzled so
+    // that "lane r reads row r" is free of bank conflicts); every worker then re-reads it from there.
+    __shared__ __align__(16) float side_tile[RUN ? 4 : kDecThreads * 32];
+    const uint64_t row0 = (uint64_t)blockIdx.x * blockDim.x;
+    if (!RUN && args.side != nullptr) {
+        // kDecThreads rows x 8 pieces = 8 pieces per thread
+#pragma unroll
+        for (uint32_t k = 0; k < 8u; ++k) {
+            const uint32_t q = threadIdx.x + (uint32_t)kDecThreads * k;       // 16-byte piece inside the CTA's block
+            const uint64_t piece = row0 * 8u + q;
+            if (piece * 4u + 4u <= args.n) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(args.side) + piece);
+                const uint32_t r = q >> 3, c = q & 7u;
+                *reinterpret_cast<float4*>(side_tile + r * 32u + ((c ^ (r & 7u)) << 2)) = v;
+            }
+        }
+        __syncthreads();
+    }
+
+    const uint64_t row = row0 + threadIdx.x;
     if (row >= args.rows) return;
     const uint64_t base = row * 32u;
     const uint64_t bucket = row / args.rows_per_bucket;
@@ -248,7 +259,7 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
         decode_partial_row<DITH, RUN>(args, row, bucket, (uint32_t)(args.n - base));
         return;
     }
-    const float* side_row = args.side ? args.side + base : nullptr;
+    const float* side_row = side_tile + (RUN ? 0u : threadIdx.x * 32u);
 
     float acc[32];
 #pragma unroll
@@ -256,11 +267,14 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
 
     for (uint32_t w = 0; w < args.W; ++w) {
         const DecWorker& wk = args.w[w];
+        uint32_t cur[8];
+        float kappa;
+        load_worker_row(wk, row, bucket, cur, kappa);
         switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
-            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, bucket, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
         }
     }
 
