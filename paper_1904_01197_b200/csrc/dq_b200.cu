@@ -5,6 +5,7 @@
 #include <atomic>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include "dq_decode.cuh"
 #include "dq_encode.cuh"
@@ -111,18 +112,39 @@ bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Launch with programmatic stream serialization allowed: the kernels of this library all begin with
+// griddepcontrol.wait (nothing is read or written before the previous kernel of the stream has completed and
+// flushed), so letting the next launch start while this one drains only hides launch latency.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), uint32_t grid, uint32_t block, size_t smem, cudaStream_t st,
+                              Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 template <int MODE, int BITS, int DITH>
 cudaError_t launch_encode_one(const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
 {
     auto k = dq::encode_kernel<BITS, MODE, DITH>;
-    static thread_local bool configured = false;
-    if (!configured) {
+    static bool configured[64] = {};        // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dq::kEncSmemBytes);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
-    k<<<grid, dq::kEncThreads, dq::kEncSmemBytes, st>>>(map, a);
-    return cudaGetLastError();
+    return launch_overlapped(k, grid, (uint32_t)dq::kEncThreads, dq::kEncSmemBytes, st, map, a);
 }
 
 template <int MODE, int DITH>
@@ -297,14 +319,15 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
     const bool d16 = (msgs[0].p.dither_bits == 16u);
     const uint32_t grid = (uint32_t)grid64;
+    cudaError_t le;
     if (running && any_nested) {
-        if (d16) dq::decode_aggregate_kernel<16, true><<<grid, dq::kDecThreads, 0, st>>>(a);
-        else dq::decode_aggregate_kernel<32, true><<<grid, dq::kDecThreads, 0, st>>>(a);
+        if (d16) le = launch_overlapped(dq::decode_aggregate_kernel<16, true>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
+        else le = launch_overlapped(dq::decode_aggregate_kernel<32, true>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
     } else {
-        if (d16) dq::decode_aggregate_kernel<16, false><<<grid, dq::kDecThreads, 0, st>>>(a);
-        else dq::decode_aggregate_kernel<32, false><<<grid, dq::kDecThreads, 0, st>>>(a);
+        if (d16) le = launch_overlapped(dq::decode_aggregate_kernel<16, false>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
+        else le = launch_overlapped(dq::decode_aggregate_kernel<32, false>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
     }
-    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    if (le != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;
 }

@@ -235,6 +235,8 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     // Side information of the CTA's 128 rows -> shared memory (coalesced loads, 16-byte pieces swizzled so
     // that "lane r reads row r" is free of bank conflicts); every worker then re-reads it from there.
     __shared__ __align__(16) float side_tile[RUN ? 4 : kDecThreads * 32];
+    grid_dependency_wait();
+    grid_dependency_launch_next();
     const uint64_t row0 = (uint64_t)blockIdx.x * blockDim.x;
     if (!RUN && args.side != nullptr) {
         // kDecThreads rows x 8 pieces = 8 pieces per thread

@@ -178,6 +178,18 @@ __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// Programmatic dependent launch: wait until the previous kernel of the stream has completed and its writes are
+// visible (a no-op when the kernel was launched normally), and allow the next kernel to begin launching.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void grid_dependency_launch_next()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // Byte offset, inside a 128-byte-swizzled tile of 128-byte rows, of 16-byte chunk `c` of row `r`.
 __device__ __forceinline__ uint32_t swz128(uint32_t r, uint32_t c)
 {

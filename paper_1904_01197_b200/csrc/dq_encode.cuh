@@ -257,7 +257,10 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31u;
 
+    grid_dependency_launch_next();
+
     if (blockIdx.x < args.plain_ctas) {
+        grid_dependency_wait();
         // plain-load part: warps take buckets round-robin over these CTAs
         for (uint64_t b = args.first_bucket + (uint64_t)blockIdx.x * kConsumerWarps + warp;
              b < args.num_buckets; b += (uint64_t)args.plain_ctas * kConsumerWarps)
@@ -275,6 +278,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
 #pragma unroll
         for (int s = 0; s < kEncStages; ++s) mbar_init(my_bar + 8u * s, 1u);
         fence_mbar_init();
+        asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmap) : "memory");
+    }
+    // nothing above touches memory that an earlier kernel of the stream may still be writing
+    grid_dependency_wait();
+    if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kEncStages; ++s) {
             const uint64_t tile = (uint64_t)first_tile + (uint64_t)s * stride;
