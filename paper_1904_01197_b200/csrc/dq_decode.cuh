@@ -1,12 +1,12 @@
 // Fused decode-and-average kernel (Algorithm 1, server steps; nested decoder equation and Algorithm 2,
-// server loop with the side information given as a vector).
+// server loop with the side information given as a vector or taken as the running mean).
 //
 // One lane owns one row = 32 consecutive elements: 32 fp32 accumulators in registers, and per worker
 // exactly `bits` packed words.  For every worker (in array order) the lane reloads that worker's words and
 // bucket scale, regenerates the 32 dithers (Philox blocks four at a time, so four dependency chains are in
 // flight), reconstructs and accumulates; the mean is written at the end.  The packed streams, the side
-// information and the output are each touched once in HBM (the side information is re-read per worker from
-// L1, which keeps it out of the register file).
+// information and the output are each touched once in HBM (the side information of a CTA's 128 rows is staged
+// in swizzled shared memory and re-read from there per worker, which keeps it out of the register file).
 //
 // The path is bound by instruction issue, not by HBM: each (element, worker) pair needs a quarter of a
 // Philox block (9.25 integer instructions) before any reconstruction arithmetic.
