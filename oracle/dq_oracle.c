@@ -115,6 +115,9 @@ float dqo_dither16_from_half(uint32_t h)
 /* dither of element i in the stream selected by dither_bits (32: one word per element; 16: see above) */
 float dqo_dither_stream(uint64_t seed, uint32_t worker, uint64_t step, uint64_t i, uint32_t dither_bits)
 {
+    /* dither_bits = 0 is the receiver that cannot reproduce the dither ("half-dithered" quantization,
+     * Section 2.1: x~_h = Q(x + u), nothing is subtracted); only the decoder accepts it */
+    if (dither_bits == 0u) return 0.0f;
     if (dither_bits == 16u)
         return dqo_dither16_from_half(dqo_dither16_half(seed, worker, step, i));
     return dqo_dither(seed, worker, step, i);
@@ -374,7 +377,8 @@ static int decode_aggregate_impl(const dqo_msg *msgs, uint32_t W, uint64_t n, ui
         int rc = check_common(m->bucket, m->bits, i0);
         if (rc) return rc;
         if (m->bucket != msgs[0].bucket) return DQO_BAD_ARG;
-        if (m->dither_bits != 32u && m->dither_bits != 16u) return DQO_BAD_ARG;
+        if (m->dither_bits != 32u && m->dither_bits != 16u &&
+            !(m->dither_bits == 0u && m->kind == DQO_KIND_DQSG)) return DQO_BAD_ARG;
         if (m->kind == DQO_KIND_DQSG) {
             uint32_t L = m->levels ? m->levels : dqo_default_levels(m->bits);
             if (L < 2u || L > (1u << m->bits)) return DQO_BAD_ARG;

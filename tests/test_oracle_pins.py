@@ -424,3 +424,27 @@ def test_oracle_rejects_bad_arguments():
         oracle.ndqsg_encode(g, 1, 0, 0, 32, 2, 5, 4.0)   # K > 2^bits
     with pytest.raises(ValueError):
         oracle.ndqsg_encode(g, 1, 0, 0, 32, 2, 4, 4.0, alpha=1.5)
+
+
+# ------------------------------------------------------------------ half-dithered decoding (Section 2.1, Lemma 1)
+def test_half_dithered_decoder_matches_stochastic_quantization_statistics():
+    # the receiver does not subtract the dither: x~_h = Q(x + u) = kappa * Delta * q.  It is unbiased and its
+    # error variance is (|x| - l/M)((l+1)/M - |x|): exactly M-level stochastic quantization (Lemma 1).
+    n, B, M = 1 << 18, 65536, 2
+    x = 0.3
+    g = np.full(n, x, dtype=np.float32)
+    g[::B] = 1.0
+    pk, sc, codes = oracle.dqsg_encode(g, SEED, 1, 2, B, 3, 2 * M + 1, want_codes=True)
+    half = oracle.decode_aggregate([oracle.Msg(pk, sc, SEED, 1, oracle.KIND_DQSG, B, 3, 2 * M + 1, dither_bits=0)], n, 2)
+    assert np.array_equal(half, ((codes - M) / M).astype(np.float32))          # kappa = 1: Delta * q
+    keep = np.ones(n, bool)
+    keep[::B] = False
+    err = half[keep].astype(np.float64) - np.float32(x)
+    d = float(np.float32(x)) - 0.0                                              # l = 0, d = x
+    assert abs(err.mean()) < 5 * math.sqrt(d * (1 / M - d) / keep.sum())
+    assert err.var() == pytest.approx(d * (1 / M - d), rel=0.03)
+    full = oracle.decode_aggregate([oracle.Msg(pk, sc, SEED, 1, oracle.KIND_DQSG, B, 3, 2 * M + 1)], n, 2)
+    assert (full[keep].astype(np.float64) - np.float32(x)).var() == pytest.approx(1 / (12 * M * M), rel=0.03)
+    with pytest.raises(ValueError):                                             # the nested decoder needs the dither
+        oracle.decode_aggregate([oracle.Msg(pk, sc, SEED, 1, oracle.KIND_NDQSG, B, 3, coarse_K=4, fine_M=2.0,
+                                            dither_bits=0)], n, 2, side_info=g)
