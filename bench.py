@@ -289,6 +289,13 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
         outs.append(torch.empty_like(st.out))
     launches = [(lambda a=msg_sets[i], b=sides[i], c=outs[i]: st.decode(a, b, c)) for i in range(sets)]
     ms = time_isolated(torch, launches, iters=12)
+    if not st.any_nested:
+        # the receiver without the dither (no random numbers): the memory-bound limit of the decoder
+        half_l = [(lambda a=msg_sets[i], c=outs[i]: dq.dqsg_decode_aggregate_half_dithered(a, n, c)) for i in range(sets)]
+        ms_h = time_isolated(torch, half_l, iters=12)
+        res["decode_aggregate_half_dithered"] = {"ms": ms_h, "bytes": per_set, "gbs": per_set / ms_h / 1e6,
+                                                 "gelem_s": n / ms_h / 1e6, "frac_hbm": per_set / ms_h / 1e6 / hbm_peak,
+                                                 "gelem_worker_s": n * cfg.W / ms_h / 1e6}
     if st.any_nested and cfg.workers[0].kind == st.DQSG:
         # Algorithm 2's own server loop on the same messages: side information = running mean, no vector read
         run_l = [(lambda a=msg_sets[i], c=outs[i]: dq.ndqsg_decode_aggregate_running(a, n, cfg.step, c))

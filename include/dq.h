@@ -132,6 +132,16 @@ dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uin
                                  void* cuda_stream);
 
 /*
+ * dqsg_decode_aggregate_half_dithered -- the receiver that cannot reproduce the dither (Section 2.1,
+ * "half-dithered quantization" x~_h = Q(x + u); by Lemma 1 this is M-level stochastic quantization): every
+ * DQSG message is reconstructed as kappa * Delta * q with nothing subtracted, and the mean is written.  No
+ * random numbers are generated, so this kernel shows the memory-bound limit of the decoder.  Seeds, worker
+ * indices and dither_bits of the messages are ignored.  Arguments as for dqsg_decode_aggregate.
+ */
+dq_status dqsg_decode_aggregate_half_dithered(const dq_msg* msgs, uint32_t W, uint64_t n, float* out_avg,
+                                              void* cuda_stream);
+
+/*
  * ndqsg_decode_aggregate_running -- the server loop of Algorithm 2 as written: the messages are visited in
  * array order; a DQSG message (group P1) is reconstructed directly; an NDQSG message (group P2) is resolved
  * against g_bar = the mean of all reconstructions before it, which is then updated with the new one ("update

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     dqsg_decode_aggregate,
     ndqsg_decode_aggregate,
     ndqsg_decode_aggregate_running,
+    dqsg_decode_aggregate_half_dithered,
     encode_workspace_bytes,
     decode_workspace_bytes,
     dqsg_encode_host,

@@ -62,6 +62,8 @@ def lib() -> C.CDLL:
         L.dqsg_decode_aggregate.restype = C.c_int
         L.ndqsg_decode_aggregate.argtypes = [pm, u32, u64, u64, vp, vp, vp, vp]
         L.ndqsg_decode_aggregate.restype = C.c_int
+        L.dqsg_decode_aggregate_half_dithered.argtypes = [pm, u32, u64, vp, vp]
+        L.dqsg_decode_aggregate_half_dithered.restype = C.c_int
         L.ndqsg_decode_aggregate_running.argtypes = [pm, u32, u64, u64, vp, vp, vp]
         L.ndqsg_decode_aggregate_running.restype = C.c_int
         L.dq_encode_workspace_bytes.argtypes = [u64, pp]; L.dq_encode_workspace_bytes.restype = u64
@@ -204,6 +206,17 @@ def ndqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, side_info
                                         _dev_ptr(out_avg, torch.float32, "out_avg"),
                                         _dev_ptr(status_word, torch.int32, "status_word"), _stream_ptr(stream)),
            "ndqsg_decode_aggregate")
+    return out_avg
+
+
+def dqsg_decode_aggregate_half_dithered(msgs: Sequence[Message], n: int, out_avg: Optional[torch.Tensor] = None,
+                                        stream=None) -> torch.Tensor:
+    """Mean of the DQSG messages reconstructed without subtracting the dither (Section 2.1, Lemma 1)."""
+    if out_avg is None:
+        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+    _check(lib().dqsg_decode_aggregate_half_dithered(_msg_array(msgs), len(msgs), n,
+                                                     _dev_ptr(out_avg, torch.float32, "out_avg"),
+                                                     _stream_ptr(stream)), "dqsg_decode_aggregate_half_dithered")
     return out_avg
 
 

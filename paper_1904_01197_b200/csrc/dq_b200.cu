@@ -254,7 +254,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
 
 dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, const float* side_info,
                         float* out_avg, uint32_t* status_word, bool allow_nested, cudaStream_t st,
-                        bool running = false)
+                        bool running = false, bool half_dithered = false)
 {
     if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
     static thread_local dq::DecodeArgs a;    // ~10 KB: keep it off the stack
@@ -268,7 +268,7 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         if (s != DQ_OK) return s;
         if (m.kind == DQ_KIND_NDQSG && !allow_nested) return DQ_ERR_INVALID_ARG;
         if (m.p.bucket != msgs[0].p.bucket) return DQ_ERR_UNSUPPORTED;
-        if ((m.p.dither_bits == 16u) != (msgs[0].p.dither_bits == 16u)) return DQ_ERR_UNSUPPORTED;
+        if (!half_dithered && (m.p.dither_bits == 16u) != (msgs[0].p.dither_bits == 16u)) return DQ_ERR_UNSUPPORTED;
         dq::DecWorker& d = a.w[w];
         d.packed = m.packed;
         d.scale = m.scale;
@@ -320,7 +320,9 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     const bool d16 = (msgs[0].p.dither_bits == 16u);
     const uint32_t grid = (uint32_t)grid64;
     cudaError_t le;
-    if (running && any_nested) {
+    if (half_dithered) {
+        le = launch_overlapped(dq::decode_aggregate_kernel<0, false>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
+    } else if (running && any_nested) {
         if (d16) le = launch_overlapped(dq::decode_aggregate_kernel<16, true>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
         else le = launch_overlapped(dq::decode_aggregate_kernel<32, true>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
     } else {
@@ -380,6 +382,13 @@ dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uin
 {
     return decode_common(msgs, W, n, step, side_info, out_avg, status_word, true,
                          static_cast<cudaStream_t>(cuda_stream));
+}
+
+dq_status dqsg_decode_aggregate_half_dithered(const dq_msg* msgs, uint32_t W, uint64_t n, float* out_avg,
+                                              void* cuda_stream)
+{
+    return decode_common(msgs, W, n, 0u, nullptr, out_avg, nullptr, false, static_cast<cudaStream_t>(cuda_stream),
+                         false, true);
 }
 
 dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, float* out_avg,

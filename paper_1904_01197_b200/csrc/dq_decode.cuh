@@ -107,7 +107,7 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, co
         uint32_t ctr[4], rnd[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) ctr[j] = (uint32_t)row * (32u / EPB) + (uint32_t)(4 * h + j);
-        philox4x32_10_xN<4>(ctr, wk.ps, rnd);
+        if (DITH != 0) philox4x32_10_xN<4>(ctr, wk.ps, rnd);
 #pragma unroll
         for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -191,7 +191,9 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t
             code &= (1u << bits) - 1u;
             uint32_t ctr[1], rnd[1][4];
             float f;
-            if (DITH == 16) {
+            if (DITH == 0) {
+                f = 1.5f;
+            } else if (DITH == 16) {
                 ctr[0] = (uint32_t)(i >> 3);
                 philox4x32_10_xN<1>(ctr, wk.ps, rnd);
                 f = dither16_f12(rnd[0][(i & 7u) >> 1], (int)(i & 1u));

@@ -105,6 +105,7 @@ __device__ __forceinline__ float dither16_f12(uint32_t word, int high)
 template <int DITH>
 __device__ __forceinline__ float dither_of(const uint32_t (&rnd)[4][4], int t)
 {
+    if (DITH == 0) return 1.5f;                      // no dither at the receiver (half-dithered decoding)
     if (DITH == 16) return dither16_f12(rnd[t >> 3][(t & 7) >> 1], t & 1);
     return dither_f12(rnd[t >> 2][t & 3]);
 }

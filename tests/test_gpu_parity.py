@@ -244,3 +244,24 @@ def test_host_buffer_entry_points(dq, oracle):
     dq.ndqsg_decode_aggregate_host(msgs, n, 4, side, out, ws)
     ref = oracle.decode_aggregate(omsgs, n, 4, side_info=side.numpy())
     assert assert_fp32_close(out.numpy(), ref, "host entry points")
+
+
+def test_half_dithered_decode_matches_oracle(dq, oracle):
+    """The receiver without the dither (Section 2.1): mean of kappa * Delta * q over the workers."""
+    import dataclasses
+    rng = np.random.default_rng(1234)
+    n, bucket, W = 3 * 8192 + 777, 1024, 5
+    specs = [WorkerSpec(DQSG, b, default_levels(b), seed=90 + b) for b in (1, 2, 3, 4, 8)]
+    omsgs, gmsgs, keep = [], [], []
+    for w, sp in enumerate(specs):
+        g = rng.standard_normal(n).astype(np.float32)
+        opk, osc = oracle_encode(oracle, g, sp, w, 6, bucket)
+        omsgs.append(oracle_msg(oracle, opk, osc, dataclasses.replace(sp, dither_bits=0), w, bucket))
+        pk = torch.from_numpy(np.concatenate([opk, np.zeros(4, np.uint32)]).view(np.int32)).cuda()
+        sc = torch.from_numpy(osc.copy()).cuda()
+        keep.append((pk, sc))
+        gmsgs.append(gpu_msg(dq, pk, sc, sp, w, bucket))
+    ref = oracle.decode_aggregate(omsgs, n, 6)
+    out = dq.dqsg_decode_aggregate_half_dithered(gmsgs, n)
+    torch.cuda.synchronize()
+    assert assert_fp32_close(out[:n].cpu().numpy(), ref, "half-dithered")
