@@ -153,6 +153,15 @@ dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_
                                          float* out_avg, uint32_t* status_word, void* cuda_stream);
 
 /*
+ * dq_code_histogram -- counts how often each code occurs in a packed message: hist[c] = number of elements
+ * whose b-bit code is c.  This is the input of the paper's rate accounting (Section 4: raw bits are
+ * log2(levels) per element, the entropy of the index stream is what an entropy coder approaches).
+ *   packed  device, dq_packed_words(n, bits) words
+ *   hist    device, uint64[2^bits], 8-byte aligned; zeroed and filled by the call
+ */
+dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, uint64_t* hist, void* cuda_stream);
+
+/*
  * Host-buffer variants.  Every data pointer (grad, out_packed, out_scale, the packed/scale pointers
  * inside msgs, side_info, out_avg) is HOST memory (pinned memory makes the copies asynchronous);
  * `workspace` is device memory of at least the stated size, 256-byte aligned, provided by the caller.

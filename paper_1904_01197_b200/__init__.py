@@ -23,6 +23,8 @@ from .binding import (  # noqa: F401
     ndqsg_decode_aggregate,
     ndqsg_decode_aggregate_running,
     dqsg_decode_aggregate_half_dithered,
+    code_histogram,
+    entropy_bits_per_element,
     encode_workspace_bytes,
     decode_workspace_bytes,
     dqsg_encode_host,

@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
         L.dqsg_decode_aggregate_half_dithered.restype = C.c_int
         L.ndqsg_decode_aggregate_running.argtypes = [pm, u32, u64, u64, vp, vp, vp]
         L.ndqsg_decode_aggregate_running.restype = C.c_int
+        L.dq_code_histogram.argtypes = [vp, u64, u32, vp, vp]
+        L.dq_code_histogram.restype = C.c_int
         L.dq_encode_workspace_bytes.argtypes = [u64, pp]; L.dq_encode_workspace_bytes.restype = u64
         L.dq_decode_workspace_bytes.argtypes = [pm, u32, u64, C.c_int]; L.dq_decode_workspace_bytes.restype = u64
         for f in (L.dqsg_encode_host, L.ndqsg_encode_host):
@@ -231,6 +233,24 @@ def ndqsg_decode_aggregate_running(msgs: Sequence[Message], n: int, step: int,
                                                 _dev_ptr(status_word, torch.int32, "status_word"),
                                                 _stream_ptr(stream)), "ndqsg_decode_aggregate_running")
     return out_avg
+
+
+def code_histogram(packed: torch.Tensor, n: int, bits: int, hist: Optional[torch.Tensor] = None,
+                   stream=None) -> torch.Tensor:
+    """hist[c] = number of elements of the packed message whose code is c (int64[2^bits] on the device)."""
+    if hist is None:
+        hist = torch.empty(1 << bits, dtype=torch.int64, device=packed.device)
+    _check(lib().dq_code_histogram(_dev_ptr(packed, torch.int32, "packed"), n, bits,
+                                   _dev_ptr(hist, torch.int64, "hist"), _stream_ptr(stream)), "dq_code_histogram")
+    return hist
+
+
+def entropy_bits_per_element(hist) -> float:
+    """Empirical entropy -sum p log2 p of a code histogram (host arithmetic on at most 256 counters)."""
+    import math
+    counts = [int(c) for c in hist.tolist()]
+    total = sum(counts)
+    return -sum(c / total * math.log2(c / total) for c in counts if c) if total else 0.0
 
 
 # ------------------------------------------------------------------------------------------ host buffers

@@ -9,6 +9,7 @@
 
 #include "dq_decode.cuh"
 #include "dq_encode.cuh"
+#include "dq_stats.cuh"
 
 namespace {
 
@@ -396,6 +397,29 @@ dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_
 {
     return decode_common(msgs, W, n, step, nullptr, out_avg, status_word, true,
                          static_cast<cudaStream_t>(cuda_stream), true);
+}
+
+dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, uint64_t* hist, void* cuda_stream)
+{
+    if (bits < 1u || bits > 8u) return DQ_ERR_INVALID_ARG;
+    if (!hist) return DQ_ERR_INVALID_ARG;
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(hist, 0, sizeof(uint64_t) << bits, st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (n == 0) return DQ_OK;
+    if (!packed) return DQ_ERR_INVALID_ARG;
+    if (!aligned16(packed) || (reinterpret_cast<uintptr_t>(hist) & 7u) != 0u) return DQ_ERR_ALIGNMENT;
+    const int sms = device_sm_count();
+    if (sms <= 0) return DQ_ERR_CUDA;
+    const uint64_t rows = (n + 31u) / 32u;
+    uint64_t grid = (rows + dq::kHistThreads - 1u) / dq::kHistThreads;
+    if (grid > (uint64_t)sms * 8u) grid = (uint64_t)sms * 8u;
+    static_assert(sizeof(unsigned long long) == sizeof(uint64_t), "histogram counters are 64-bit");
+    if (launch_overlapped(dq::code_histogram_kernel, (uint32_t)grid, (uint32_t)dq::kHistThreads, 0, st, packed, n,
+                          bits, reinterpret_cast<unsigned long long*>(hist)) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return DQ_OK;
 }
 
 // ------------------------------------------------------------------------------------------------ host buffers

@@ -265,3 +265,19 @@ def test_half_dithered_decode_matches_oracle(dq, oracle):
     out = dq.dqsg_decode_aggregate_half_dithered(gmsgs, n)
     torch.cuda.synchronize()
     assert assert_fp32_close(out[:n].cpu().numpy(), ref, "half-dithered")
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 5, 8])
+def test_code_histogram_matches_oracle_counts(dq, oracle, bits):
+    rng = np.random.default_rng(4321 + bits)
+    n = 300_000 + 19
+    g = rng.standard_normal(n).astype(np.float32)
+    spec = WorkerSpec(DQSG, bits, default_levels(bits), seed=66)
+    pk, sc, opk, osc = _check_encode(dq, oracle, g, spec, 0, 3, 2048)
+    want = np.bincount(oracle.unpack(opk, n, bits), minlength=1 << bits)
+    hist = dq.code_histogram(pk.contiguous(), n, bits)
+    torch.cuda.synchronize()
+    assert np.array_equal(hist.cpu().numpy(), want)
+    H = dq.entropy_bits_per_element(hist)
+    p = want[want > 0] / n
+    assert abs(H + (p * np.log2(p)).sum()) < 1e-9

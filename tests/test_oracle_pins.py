@@ -448,3 +448,20 @@ def test_half_dithered_decoder_matches_stochastic_quantization_statistics():
     with pytest.raises(ValueError):                                             # the nested decoder needs the dither
         oracle.decode_aggregate([oracle.Msg(pk, sc, SEED, 1, oracle.KIND_NDQSG, B, 3, coarse_K=4, fine_M=2.0,
                                             dither_bits=0)], n, 2, side_info=g)
+
+
+# ------------------------------------------------------------------ index statistics (rate after entropy coding)
+def test_ternary_index_distribution_and_entropy_for_uniform_input():
+    # x ~ U[-1, 1], kappa = 1, M = 1: P(q = +1) = E[max(x, 0)] = 1/4 = P(q = -1), P(q = 0) = 1/2 (Appendix A),
+    # so the index stream carries 1.5 bits per element, below the raw log2(3) of the raw-bits table.
+    rng = np.random.default_rng(77)
+    n, B = 1 << 18, 65536
+    g = rng.uniform(-1, 1, n).astype(np.float32)
+    g[::B] = 1.0
+    pk, sc = oracle.dqsg_encode(g, SEED, 0, 1, B, 2, 3)
+    hist = np.bincount(oracle.unpack(pk, n, 2), minlength=4)
+    assert hist.sum() == n and hist[3] == 0
+    p = hist[:3] / n
+    assert np.allclose(p, [0.25, 0.5, 0.25], atol=5 * math.sqrt(0.25 / n))
+    H = -(p * np.log2(p)).sum()
+    assert H == pytest.approx(1.5, abs=0.01) and H < math.log2(3)
