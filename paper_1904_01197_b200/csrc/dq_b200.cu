@@ -208,26 +208,28 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     }
     fill_philox(a.ps, seed, worker, step);
 
-    // power-of-two buckets up to 8192: whole tiles of 8192 elements go through the tile path of the kernel,
-    // the rest (and every other bucket size) through its plain-load part, in the same launch
+    // power-of-two buckets up to 8192: whole work units (a bucket, or 1024 elements for smaller buckets) go
+    // through the tile path of the kernel, the rest (and every other bucket size) through its plain-load part,
+    // in the same launch
     const int sms = device_sm_count();
     if (sms <= 0) return DQ_ERR_CUDA;
     const uint32_t B = p->bucket;
-    const uint32_t T = (uint32_t)dq::kTileRows * 32u;
-    uint64_t tiles = (is_pow2(B) && B <= T) ? n / T : 0u;
+    const uint32_t U = (B < 1024u) ? 1024u : B;                     // elements per work unit
+    uint64_t tiles = (is_pow2(B) && B <= 8192u) ? n / U : 0u;       // whole units
     if (tiles > 0xFFFFFFFFull) return DQ_ERR_UNSUPPORTED;
     CUtensorMap map;
     std::memset(&map, 0, sizeof(map));
+    const uint32_t wpb = (B < 1024u) ? 1u : (B / 1024u);
     if (tiles > 0) {
-        if (!make_row_map(&map, grad, tiles * dq::kTileRows, 32u)) return DQ_ERR_CUDA;
-        a.num_tiles = (uint32_t)tiles;
+        if (!make_row_map(&map, grad, tiles * (U / 32u), 32u)) return DQ_ERR_CUDA;
+        a.num_units = (uint32_t)tiles;
         a.lanes_per_bucket = (B < 1024u) ? (B / 32u) : 32u;
-        a.warps_per_bucket = (B < 1024u) ? 1u : (B / 1024u);
+        a.warps_per_bucket = wpb;
         uint32_t lg = 0;
         while ((1u << lg) < B) ++lg;
         a.bucket_log2 = lg;
     }
-    a.first_bucket = tiles * (T / B);
+    a.first_bucket = tiles * (U / B);
     const uint64_t rest = a.num_buckets - a.first_bucket;
     const uint32_t slots = (uint32_t)dq::kEncCtasPerSm * (uint32_t)sms;   // resident CTAs
     uint32_t plain = 0;
@@ -241,7 +243,9 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     uint32_t tile_ctas = 0;
     if (tiles > 0) {
         const uint32_t room = (slots > plain) ? (slots - plain) : 1u;
-        tile_ctas = (uint32_t)(tiles < room ? tiles : room);
+        const uint64_t groups_per_cta = (uint64_t)dq::kConsumerWarps / wpb;
+        const uint64_t want_ctas = (tiles + groups_per_cta - 1u) / groups_per_cta;
+        tile_ctas = (uint32_t)(want_ctas < room ? want_ctas : room);
     }
     cudaError_t e;
     const bool d16 = (p->dither_bits == 16u);

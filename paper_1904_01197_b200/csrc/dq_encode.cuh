@@ -45,7 +45,7 @@ struct EncodeArgs {
     uint64_t first_bucket;   // first bucket of the plain-load part
     uint64_t num_buckets;    // total buckets of the gradient
     uint64_t num_words;      // total packed words of the gradient
-    uint32_t num_tiles;      // whole 8192-element tiles taken by the tile path
+    uint32_t num_units;      // work units of the tile path: max(B, 1024) elements each (see encode_kernel)
     uint32_t plain_ctas;     // the first plain_ctas CTAs run the plain-load part, the rest walk over the tiles
     uint32_t bucket;         // B
     uint32_t bucket_log2;    // log2(B) on the tile path
@@ -241,8 +241,8 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
 // The encode kernel.  Grid = CTAs for the plain-load part (scheduled first) + persistent tile CTAs.
 // Block = 8 warps.  Dynamic shared memory = kEncSmemBytes.
 //
-// Tile path: a CTA walks over tiles of 8192 elements; warp w owns rows [32 w, 32 w + 32) of each tile and
-// runs its own two-stage pipeline: its lane 0 issues the 4 KB tile copy for the tile after next as soon as
+// Tile path: the warps of a CTA form groups (one group per bucket position); a group walks over work units
+// and each of its warps owns 32 rows of every unit and runs its own two-stage pipeline: its lane 0 issues the 4 KB tile copy for the tile after next as soon as
 // the warp has taken the current rows into registers, so a copy is always in flight while the warp
 // quantizes, and no warp ever waits for another one except the warps that share a bucket (named barrier).
 // ---------------------------------------------------------------------------------------------------
@@ -271,8 +271,16 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t my_smem = smem_base + warp * (uint32_t)(kEncStages * kWarpTileBytes);
     const uint32_t my_bar = smem_u32(&bar_full[warp][0]);
-    const uint32_t stride = gridDim.x - args.plain_ctas;
-    const uint32_t first_tile = blockIdx.x - args.plain_ctas;
+    // Work unit = the rows of one bucket (B >= 1024: B / 1024 warps work on it together) or 1024 elements
+    // (smaller buckets: one warp).  The groups of all tile CTAs take units round-robin, which spreads the work
+    // over the SMs to within one unit.
+    const uint32_t wpb = args.warps_per_bucket;      // warps sharing a bucket (1, 2, 4, 8)
+    const uint32_t group = warp / wpb;               // group of this warp inside the CTA
+    const uint32_t groups_per_cta = (uint32_t)kConsumerWarps / wpb;
+    const uint32_t stride = (gridDim.x - args.plain_ctas) * groups_per_cta;
+    const uint32_t first_tile = (blockIdx.x - args.plain_ctas) * groups_per_cta + group;
+    const uint32_t unit_rows = wpb * 32u;
+    const uint32_t row_in_unit = (warp % wpb) * 32u;
 
     if (lane == 0) {
 #pragma unroll
@@ -286,21 +294,19 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
 #pragma unroll
         for (int s = 0; s < kEncStages; ++s) {
             const uint64_t tile = (uint64_t)first_tile + (uint64_t)s * stride;
-            if (tile < args.num_tiles) {
+            if (tile < args.num_units) {
                 mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
                 tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
-                              (int32_t)(tile * kTileRows + warp * 32u));
+                              (int32_t)(tile * unit_rows + row_in_unit));
             }
         }
     }
     __syncwarp();
 
     const uint32_t swz = lane & 7u;                  // (row & 7): the warp's rows start at a multiple of 32
-    const uint32_t wpb = args.warps_per_bucket;      // warps sharing a bucket (1, 2, 4, 8)
-    const uint32_t group = warp / wpb;               // bucket of this warp inside the tile, when B >= 1024
     bool gave_up = false;
     uint32_t k = 0;
-    for (uint64_t tile = first_tile; tile < args.num_tiles; tile += stride, ++k) {
+    for (uint64_t tile = first_tile; tile < args.num_units; tile += stride, ++k) {
         const uint32_t s = k % kEncStages;
         const uint32_t use = k / kEncStages;
         if (!mbar_wait_bounded(my_bar + 8u * s, use & 1u, gave_up ? 1u : (1u << 22))) {
@@ -330,13 +336,13 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         __syncwarp();
         if (lane == 0) {
             const uint64_t next = tile + (uint64_t)kEncStages * stride;
-            if (next < args.num_tiles) {
+            if (next < args.num_units) {
                 mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
                 tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
-                              (int32_t)(next * kTileRows + warp * 32u));
+                              (int32_t)(next * unit_rows + row_in_unit));
             }
         }
-        const uint32_t row = (uint32_t)tile * kTileRows + warp * 32u + lane;   // row index in the gradient (< 2^29)
+        const uint32_t row = (uint32_t)tile * unit_rows + row_in_unit + lane;   // row index in the gradient (< 2^29)
         if (wpb > 1u) {
             if (lane == 0) warp_max[k & 1u][warp] = mx;
             named_bar_sync(1u + group, wpb * 32u);
