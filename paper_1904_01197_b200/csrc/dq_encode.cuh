@@ -5,12 +5,13 @@
 // `bits` 32-bit words of the bit stream.  One lane quantizes and packs a whole row, so no lane ever shares a
 // packed word with another lane and no shuffles are needed for packing.
 //
-// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight warps walk over tiles of 8192
-// elements (256 rows).  Every warp owns 32 rows of each tile and keeps its own two-stage shared-memory
-// pipeline filled with asynchronous 2-D tile copies (128-byte swizzle, which makes "lane r reads row r" free
-// of bank conflicts): it takes its rows of a stage into registers, re-arms the stage with the copy for the
-// tile after next, reduces max|g| over its bucket (shuffles inside the warp, a named barrier between the
-// warps that share a bucket) and then quantizes from registers.  The gradient is read from HBM exactly once.
+// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight warps.  The warps of a CTA form
+// groups of B/1024 warps (one warp for smaller buckets); the groups of all CTAs take work units -- one bucket,
+// or 1024 elements -- round-robin.  Every warp owns 32 rows of each unit and keeps its own two-stage
+// shared-memory pipeline filled with asynchronous 2-D tile copies (128-byte swizzle, which makes "lane r reads
+// row r" free of bank conflicts): it takes its rows of a stage into registers, re-arms the stage with the copy
+// for the unit after next, reduces max|g| over its bucket (shuffles inside the warp, a named barrier between
+// the warps that share a bucket) and then quantizes from registers.  The gradient is read from HBM exactly once.
 //
 // Everything else -- other bucket sizes, the part of the vector past the last whole tile, the ragged end --
 // is handled by plain-load code, one warp per bucket, in extra CTAs of the same launch.
@@ -22,7 +23,7 @@ namespace dq {
 
 enum EncMode : int { kEncDqsg = 0, kEncNdqsgPow2 = 1, kEncNdqsgAnyK = 2 };
 
-constexpr int kTileRows = 256;                     // rows per tile (8192 elements, 32 KB)
+constexpr int kTileRows = 256;                     // rows a CTA holds per pipeline stage (8 warps x 32 rows, 32 KB)
 constexpr int kTileBytes = kTileRows * 128;
 constexpr int kConsumerWarps = kTileRows / 32;     // one row per lane
 constexpr int kWarpTileBytes = 32 * 128;           // the 32 rows of a tile that one warp owns
