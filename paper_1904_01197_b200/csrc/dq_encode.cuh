@@ -52,6 +52,7 @@ struct EncodeArgs {
     uint32_t bucket_log2;    // log2(B) on the tile path
     uint32_t lanes_per_bucket;  // B / 32 when B < 1024, else 32
     uint32_t warps_per_bucket;  // B / 1024 when B >= 1024, else 1
+    uint32_t pair_in_time;      // B == 2048: one warp handles both halves of a bucket (units are buckets)
     float gain_num;          // DQSG: s = (L-1)/2;  NDQSG: A = alpha * M1
     float shift;             // DQSG: s
     float kmax;              // DQSG: L - 1
@@ -294,11 +295,12 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kEncStages; ++s) {
-            const uint64_t tile = (uint64_t)first_tile + (uint64_t)s * stride;
+            // first copies: the next two units of this warp, or (pair mode) the two halves of its first bucket
+            const uint64_t tile = args.pair_in_time ? (uint64_t)first_tile : (uint64_t)first_tile + (uint64_t)s * stride;
+            const uint64_t row0 = args.pair_in_time ? tile * 64u + (uint64_t)s * 32u : tile * unit_rows + row_in_unit;
             if (tile < args.num_units) {
                 mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
-                tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
-                              (int32_t)(tile * unit_rows + row_in_unit));
+                tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s, (int32_t)row0);
             }
         }
     }
@@ -307,6 +309,74 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     const uint32_t swz = lane & 7u;                  // (row & 7): the warp's rows start at a multiple of 32
     bool gave_up = false;
     uint32_t k = 0;
+
+    if (args.pair_in_time) {
+        // B = 2048: one warp handles the whole bucket as two consecutive 1024-element halves, one per stage, so
+        // no other warp is involved.  The second half only has to have landed (it was requested a whole unit
+        // earlier) for its maximum to be read from shared memory before the first half is quantized.
+        for (uint64_t pair = first_tile; pair < args.num_units; pair += stride, ++k) {
+            const uint32_t par = k & 1u;
+            float x[32];
+            float mx = 0.0f;
+#pragma unroll 1
+            for (uint32_t half = 0; half < 2u; ++half) {
+                const uint32_t stage_addr = my_smem + half * kWarpTileBytes + lane * 128u;
+                if (half == 0u) {
+                    if (!mbar_wait_bounded(my_bar, par, gave_up ? 1u : (1u << 22)) ||
+                        !mbar_wait_bounded(my_bar + 8u, par, gave_up ? 1u : (1u << 22))) {
+                        gave_up = true;
+                        if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
+                    }
+                    // maximum of the second half, straight from shared memory
+                    const uint32_t other = my_smem + kWarpTileBytes + lane * 128u;
+#pragma unroll
+                    for (uint32_t c = 0; c < 8; ++c) {
+                        float4 v;
+                        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                                     : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                     : "r"(other + ((c ^ swz) << 4))
+                                     : "memory");
+                        mx = max3_abs(max3_abs(mx, v.x, v.y), v.z, v.w);
+                    }
+                }
+#pragma unroll
+                for (uint32_t c = 0; c < 8; ++c) {
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                                 : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
+                                 : "r"(stage_addr + ((c ^ swz) << 4))
+                                 : "memory");
+                }
+                if (half == 0u) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) mx = max3_abs(mx, x[e], x[e + 1]);
+#pragma unroll
+                    for (uint32_t off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+                    if (lane == 0) args.scale[pair] = mx;
+                } else {
+                    uint32_t sink = 0u;                 // all loads of this half have completed after this
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) sink ^= __float_as_uint(x[4 * c]);
+                    asm volatile("" ::"r"(sink));
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    const uint64_t next = pair + stride;
+                    if (next < args.num_units) {
+                        mbar_expect_tx(my_bar + 8u * half, (uint32_t)kWarpTileBytes);
+                        tma_load_rows(my_smem + half * kWarpTileBytes, &tmap, my_bar + 8u * half,
+                                      (int32_t)(next * 64u + half * 32u));
+                    }
+                }
+                const float a = bucket_gain(args.gain_num, mx);
+                const uint32_t row = (uint32_t)pair * 64u + half * 32u + lane;
+                uint32_t out[BITS];
+                encode_row<BITS, MODE, DITH>(x, row, a, args, out);
+                store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
+            }
+        }
+        return;
+    }
+
     for (uint64_t tile = first_tile; tile < args.num_units; tile += stride, ++k) {
         const uint32_t s = k % kEncStages;
         const uint32_t use = k / kEncStages;
