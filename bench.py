@@ -42,9 +42,9 @@ DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
 NCU_TRAFFIC = {
-    ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_613_504,    # profiles/encode_kernel_ndqsg_resnet50.md
-    ("encode", "ndqsg_resnet50", 25_557_032, 3): 106_926_336,
-    ("decode", "ndqsg_resnet50", 25_557_032): 219_364_608,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
+    ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_689_280,    # profiles/encode_kernel_ndqsg_resnet50.md
+    ("encode", "ndqsg_resnet50", 25_557_032, 3): 105_917_696,
+    ("decode", "ndqsg_resnet50", 25_557_032): 219_741_696,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
 }
 
 
