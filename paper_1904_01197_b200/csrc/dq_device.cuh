@@ -168,11 +168,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     return false;
 }
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
 // Named barrier over `threads` threads (a multiple of 32); id 1..15 (0 is __syncthreads).
 __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
 {
@@ -189,12 +184,6 @@ __device__ __forceinline__ void grid_dependency_wait()
 __device__ __forceinline__ void grid_dependency_launch_next()
 {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-}
-
-// Byte offset, inside a 128-byte-swizzled tile of 128-byte rows, of 16-byte chunk `c` of row `r`.
-__device__ __forceinline__ uint32_t swz128(uint32_t r, uint32_t c)
-{
-    return r * 128u + ((c ^ (r & 7u)) << 4);
 }
 
 }  // namespace dq
