@@ -39,6 +39,11 @@ SM_COUNT, ISSUE_PER_SM_CLK, LANES = 148, 4, 32           # ALU-issue ceiling: SM
 # Algorithmic lane-instructions: ~22 per (element, worker) + ~10 per element for the fused decode,
 # ~24 per element for the encode.
 DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 24.0
+# Executed lane-instructions per (element, worker) of the fused decode on the ResNet-50-sized workload, split into
+# the half-rate class (integer, logic, IMAD, shifts, branches, loads) and fp32, from the opcode counters in
+# profiles/decode_aggregate_kernel_ndqsg_resnet50.md: the issue ceiling of that mix is
+# schedulers x lanes x clock / (2 * half_rate + fp32).
+DEC_MIX = {32: (17.0, 8.8), 16: (13.2, 8.8)}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
 NCU_TRAFFIC = {
@@ -569,6 +574,12 @@ def main():
                                "traffic": kd["traffic"],
                                "peak_source": "148 SMs x 4 schedulers x 32 lanes x max SM clock",
                                "hbm_gbs": kd["gbs"], "frac_hbm": kd["frac_hbm"], "launches_per_step": 1}
+            mix = DEC_MIX.get(cfg.workers[0].dither_bits)
+            if mix and cfg.name == "ndqsg_resnet50":
+                ceiling = SM_COUNT * ISSUE_PER_SM_CLK * LANES * sm_max_mhz * 1e6 / (2.0 * mix[0] + mix[1])
+                roofline_decode["issue_mix"] = {"half_rate_instr_per_unit": mix[0], "fp32_instr_per_unit": mix[1],
+                                                "ceiling_gelem_worker_s": ceiling / 1e9,
+                                                "frac_of_ceiling": kd["gelem_worker_s"] * 1e9 / ceiling}
             if kd["ms"] >= count[dom_enc] * ke["ms"]:
                 roofline = roofline_decode
             else:
