@@ -86,19 +86,40 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, const PhiloxStream& p
     out[0] = o[0][0]; out[1] = o[0][1]; out[2] = o[0][2]; out[3] = o[0][3];
 }
 
-// 32 random bits -> f in [1, 2) on the odd grid; the dither in fine-step units is f - 1.5 (exact).
+// Dither values without an integer-to-float conversion and with a single integer instruction: the 22 random
+// bits j = x >> 10, read as a float, are the subnormal j * 2^-149; one multiply-add scales them by 2^127 and
+// adds the offset, and since the result lies on the grid of step 2^-23 it is exact.  (Integer and logic
+// instructions cost about twice the issue bandwidth of fp32 ones on this GPU.)
+//   f     = 1 + (2j+1) 2^-23              in [1, 2): the dither in fine-step units is f - 1.5
+//   delta = (2j+1) 2^-23 - 1/2            the dither itself
+constexpr float kTwo127 = 1.7014118346046923e38f;      // 2^127
+constexpr float kTwo125 = 4.2535295865117308e37f;      // 2^125
+
 __device__ __forceinline__ float dither_f12(uint32_t x)
 {
-    return __uint_as_float((x >> 9) | 0x3F800001u);
+    return __fmaf_rn(__uint_as_float(x >> 10), kTwo127, 1.00000011920928955078125f);      // 1 + 2^-23
 }
 
-// 16-bit stream: half-word h -> f = 1 + (2h+1) 2^-17 in [1, 2); the dither is again f - 1.5 (exact).
+__device__ __forceinline__ float dither_delta(uint32_t x)
+{
+    return __fmaf_rn(__uint_as_float(x >> 10), kTwo127, -0.49999988079071044921875f);     // -(1/2 - 2^-23)
+}
+
+// 16-bit stream: half-word h -> f = 1 + (2h+1) 2^-17, delta = (2h+1) 2^-17 - 1/2.  One byte permutation puts
+// h into bits 8..23 (the subnormal or small normal number h * 2^-141); the multiply-add scales by 2^125.
+__device__ __forceinline__ float half_word_as_small_float(uint32_t word, int high)
+{
+    return __uint_as_float(__byte_perm(word, 0u, high ? 0x4324u : 0x4104u));
+}
+
 __device__ __forceinline__ float dither16_f12(uint32_t word, int high)
 {
-    // h * 128 + 0x3F800040: the half-word lands in mantissa bits 7..22 and bit 6 makes the grid odd; the two
-    // fields do not overlap, so the multiply-add is the same as shift-and-or but needs a single constant.
-    const uint32_t h = high ? (word >> 16) : (word & 0xFFFFu);
-    return __uint_as_float(h * 128u + 0x3F800040u);
+    return __fmaf_rn(half_word_as_small_float(word, high), kTwo125, 1.00000762939453125f);   // 1 + 2^-17
+}
+
+__device__ __forceinline__ float dither16_delta(uint32_t word, int high)
+{
+    return __fmaf_rn(half_word_as_small_float(word, high), kTwo125, -0.49999237060546875f);  // -(1/2 - 2^-17)
 }
 
 // f of element t (0 .. 4*EPB-1) of a group of four Philox blocks; EPB = elements per block (4 or 8).
@@ -108,6 +129,14 @@ __device__ __forceinline__ float dither_of(const uint32_t (&rnd)[4][4], int t)
     if (DITH == 0) return 1.5f;                      // no dither at the receiver (half-dithered decoding)
     if (DITH == 16) return dither16_f12(rnd[t >> 3][(t & 7) >> 1], t & 1);
     return dither_f12(rnd[t >> 2][t & 3]);
+}
+
+// The dither itself (encoder side).
+template <int DITH>
+__device__ __forceinline__ float dither_delta_of(const uint32_t (&rnd)[4][4], int t)
+{
+    if (DITH == 16) return dither16_delta(rnd[t >> 3][(t & 7) >> 1], t & 1);
+    return dither_delta(rnd[t >> 2][t & 3]);
 }
 
 // Round-to-nearest-even of |w| < 2^22 by adding 1.5 * 2^23: the integer lands in the low mantissa bits.

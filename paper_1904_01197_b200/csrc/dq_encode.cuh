@@ -83,10 +83,8 @@ __device__ __forceinline__ void put_bits(uint32_t (&out)[BITS], int bit, int nbi
 
 // DQSG: the rounded, clamped index of one element as an exact small float (0 .. L-1).
 //   v = fma(g, a, delta);  w = v + s;  k = clamp(rint(w), 0, L-1)   (clamping before rounding gives the same k)
-// f = dither + 1.5 in [1, 2).
-__device__ __forceinline__ float dqsg_index_f(float x, float a, float f, const EncodeArgs& args)
+__device__ __forceinline__ float dqsg_index_f(float x, float a, float delta, const EncodeArgs& args)
 {
-    const float delta = __fadd_rn(f, -1.5f);                              // exact
     const float v = __fmaf_rn(x, a, delta);
     float w = __fadd_rn(v, args.shift);
     w = fminf(fmaxf(w, 0.0f), args.kmax);
@@ -94,9 +92,8 @@ __device__ __forceinline__ float dqsg_index_f(float x, float a, float f, const E
 }
 
 // NDQSG: bit pattern kMagicBits + q1 (two's complement in the low bits) of one element.
-__device__ __forceinline__ uint32_t ndqsg_index_bits(float x, float a, float f)
+__device__ __forceinline__ uint32_t ndqsg_index_bits(float x, float a, float delta)
 {
-    const float delta = __fadd_rn(f, -1.5f);
     const float v = __fmaf_rn(x, a, delta);
     return __float_as_uint(__fadd_rn(v, kMagic));
 }
@@ -135,7 +132,7 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, f
 #pragma unroll
             for (int t = PASS - 1; t >= 0; --t) {
                 const int idx = PASS * h + t;
-                const uint32_t tb = ndqsg_index_bits(x[idx], a, dither_of<DITH>(rnd, t));
+                const uint32_t tb = ndqsg_index_bits(x[idx], a, dither_delta_of<DITH>(rnd, t));
                 unit = __funnelshift_l(tb << (32 - BITS), (idx % U == U - 1) ? 0u : unit, BITS);
                 if (idx % U == 0) put_bits<BITS>(out, idx * BITS, U * BITS, unit);
             }
@@ -143,9 +140,9 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, f
 #pragma unroll
             for (int t = 0; t < PASS; ++t) {
                 const int idx = PASS * h + t;
-                const float f = dither_of<DITH>(rnd, t);
+                const float delta = dither_delta_of<DITH>(rnd, t);
                 if (MODE == kEncDqsg) {
-                    const float kf = dqsg_index_f(x[idx], a, f, args);
+                    const float kf = dqsg_index_f(x[idx], a, delta, args);
                     const int pos = idx % G;                               // position inside the group
                     grp = (pos == 0) ? kf : __fmaf_rn(kf, (float)(1u << (BITS * pos)), grp);   // exact
                     if (pos == G - 1 || idx == 31) {
@@ -154,7 +151,7 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, f
                         put_bits<BITS>(out, first * BITS, (pos + 1) * BITS, gb);
                     }
                 } else {
-                    const uint32_t tb = ndqsg_index_bits(x[idx], a, f);
+                    const uint32_t tb = ndqsg_index_bits(x[idx], a, delta);
                     uint32_t code;
                     if (MODE == kEncNdqsgPow2) code = tb & (args.K - 1u);
                     else code = (tb - kMagicBits + args.K_offset) % args.K;   // q1 + positive multiple of K
