@@ -11,7 +11,9 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "lib" / "libdq_b200.so"
 SOURCES = [CSRC / "dq_b200.cu"]
-DEPS = sorted(CSRC.glob("*.cu*")) + [ROOT / "include" / "dq.h"]
+PROBE_SOURCE = CSRC / "issue_probe.cu"          # stand-alone program, see issue_probe.py
+PROBE = PKG / "lib" / "dq_issue_probe"
+DEPS = sorted(f for f in CSRC.glob("*.cu*") if f != PROBE_SOURCE) + [ROOT / "include" / "dq.h"]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3",
@@ -50,5 +52,18 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
+def build_probe(force: bool = False) -> Path:
+    """Compiles the issue-cost probe (a stand-alone executable that uses no library code)."""
+    if not force and PROBE.exists() and PROBE.stat().st_mtime >= PROBE_SOURCE.stat().st_mtime:
+        return PROBE
+    PROBE.parent.mkdir(parents=True, exist_ok=True)
+    tmp = PROBE.with_suffix(f".{os.getpid()}.tmp")
+    subprocess.run([nvcc_path(), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+                    "-cudart", "static", "-o", str(tmp), str(PROBE_SOURCE)], check=True)
+    os.replace(tmp, PROBE)
+    return PROBE
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_probe(force="--force" in sys.argv))
