@@ -85,6 +85,12 @@ def lib():
         L.dqo_pack.restype = None
         L.dqo_unpack.argtypes = [u32p, C.c_uint64, C.c_uint32, u32p]
         L.dqo_unpack.restype = None
+        L.dqo_ternary_bytes.argtypes = [C.c_uint64]
+        L.dqo_ternary_bytes.restype = C.c_uint64
+        L.dqo_ternary_pack.argtypes = [u32p, C.c_uint64, C.POINTER(C.c_uint8)]
+        L.dqo_ternary_pack.restype = None
+        L.dqo_ternary_unpack.argtypes = [C.POINTER(C.c_uint8), C.c_uint64, u32p]
+        L.dqo_ternary_unpack.restype = None
         L.dqo_dqsg_encode.argtypes = [f32p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64,
                                       C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32, u32p, f32p, i32p, C.c_int]
         L.dqo_dqsg_encode.restype = C.c_int
@@ -189,6 +195,36 @@ def unpack(words: np.ndarray, n: int, bits: int) -> np.ndarray:
     out = np.zeros(n, dtype=np.uint32)
     lib().dqo_unpack(_p(words, C.c_uint32), n, bits, _p(out, C.c_uint32))
     return out
+
+
+def ternary_bytes(n: int) -> int:
+    return int(lib().dqo_ternary_bytes(n))
+
+
+def ternary_pack(code: np.ndarray) -> np.ndarray:
+    """Five ternary codes per byte (radix-3 container of a three-level message)."""
+    code = np.ascontiguousarray(code, dtype=np.uint32)
+    out = np.zeros(ternary_bytes(code.size), dtype=np.uint8)
+    lib().dqo_ternary_pack(_p(code, C.c_uint32), code.size, _p(out, C.c_uint8))
+    return out
+
+
+def ternary_unpack(data: np.ndarray, n: int) -> np.ndarray:
+    data = np.ascontiguousarray(data, dtype=np.uint8)
+    assert data.size >= ternary_bytes(n)
+    out = np.zeros(n, dtype=np.uint32)
+    lib().dqo_ternary_unpack(_p(data, C.c_uint8), n, _p(out, C.c_uint32))
+    return out
+
+
+def ternary_pack_stream(words: np.ndarray, n: int) -> np.ndarray:
+    """The radix-3 container of a 2-bit packed three-level message."""
+    return ternary_pack(unpack(words, n, 2))
+
+
+def ternary_unpack_stream(data: np.ndarray, n: int) -> np.ndarray:
+    """Back to the 2-bit packed stream."""
+    return pack(ternary_unpack(data, n), 2)
 
 
 def _check(rc: int, what: str):

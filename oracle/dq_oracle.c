@@ -197,6 +197,44 @@ void dqo_unpack(const uint32_t *words, uint64_t n, uint32_t bits, uint32_t *code
 }
 
 /* ------------------------------------------------------------------------
+ * Radix-3 container for three-level messages (the paper's raw-bit count for
+ * DQSGD with M = 1 is log2(3) = 1.585 bits per element, Section 4, raw-bits
+ * table): byte k carries the five ternary codes 5k .. 5k+4 as the number
+ *     t_{5k} + 3 t_{5k+1} + 9 t_{5k+2} + 27 t_{5k+3} + 81 t_{5k+4}   (< 243),
+ * codes past the end of the vector counting as 0; 8/5 = 1.6 bits per element.
+ * A three-level message only holds the codes 0, 1, 2; a code above 2 is
+ * stored as 2.
+ * ---------------------------------------------------------------------- */
+uint64_t dqo_ternary_bytes(uint64_t n) { return (n + 4u) / 5u; }
+
+void dqo_ternary_pack(const uint32_t *code, uint64_t n, uint8_t *bytes)
+{
+    uint64_t nb = dqo_ternary_bytes(n);
+    for (uint64_t k = 0; k < nb; ++k) {
+        uint32_t v = 0, weight = 1;
+        for (uint32_t q = 0; q < 5u; ++q) {
+            uint64_t i = 5u * k + q;
+            uint32_t t = (i < n) ? code[i] : 0u;
+            if (t > 2u)
+                t = 2u;
+            v += t * weight;
+            weight *= 3u;
+        }
+        bytes[k] = (uint8_t)v;
+    }
+}
+
+void dqo_ternary_unpack(const uint8_t *bytes, uint64_t n, uint32_t *code)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        uint32_t v = bytes[i / 5u];
+        for (uint32_t q = 0; q < (uint32_t)(i % 5u); ++q)
+            v /= 3u;
+        code[i] = v % 3u;
+    }
+}
+
+/* ------------------------------------------------------------------------
  * Per-bucket scale: kappa_j = max |g_i| over the bucket (kappa = ||g||_inf of
  * Eq. (DQSG), one per partition as in the partitioning paragraph of 3.1).
  * ---------------------------------------------------------------------- */

@@ -10,7 +10,8 @@ import pytest
 
 ROOT = Path(__file__).resolve().parent.parent
 SRC = (ROOT / "oracle" / "dq_oracle.c").read_text()
-PIN_FILES = ["tests/test_oracle_pins.py", "tests/test_oracle_dither16.py", "tests/test_oracle_running_mean.py"]
+PIN_FILES = ["tests/test_oracle_pins.py", "tests/test_oracle_dither16.py", "tests/test_oracle_running_mean.py",
+             "tests/test_oracle_ternary.py"]
 
 MUTANTS = [
     ("philox multipliers swapped", "(uint64_t)0xD2511F53u * (uint64_t)c0", "(uint64_t)0xCD9E8D57u * (uint64_t)c0"),
@@ -32,6 +33,9 @@ MUTANTS = [
     ("half-words swapped in the 16-bit stream", "return (i & 1u) ? (word >> 16) : (word & 0xFFFFu);", "return (i & 1u) ? (word & 0xFFFFu) : (word >> 16);"),
     ("16-bit grid off centre", "(float)(2u * h + 1u) * 0x1p-17f - 0.5f", "(float)(2u * h) * 0x1p-17f - 0.5f"),
     ("running mean counts one worker too many", "acc * (1.0f / (float)w)", "acc * (1.0f / (float)(w + 1u))"),
+    ("ternary digit weights", "weight *= 3u;", "weight *= 4u;"),
+    ("ternary digits read in the wrong order", "q < (uint32_t)(i % 5u); ++q)", "q < 4u - (uint32_t)(i % 5u); ++q)"),
+    ("ternary container drops the last partial byte", "return (n + 4u) / 5u;", "return n / 5u;"),
     ("scalar quantizer truncates", "return Delta * nearbyint(v / Delta);", "return Delta * floor(v / Delta);"),
     ("nested scalar decoder drops the coarse term", "return y + alpha * (r - dqo_Q(r, Delta2));", "return y + alpha * r;"),
 ]
