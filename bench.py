@@ -311,6 +311,18 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
                                                 "gelem_s": n / ms_run / 1e6,
                                                 "frac_hbm": by_run / ms_run / 1e6 / hbm_peak,
                                                 "gelem_worker_s": n * cfg.W / ms_run / 1e6}
+    tern = [w for w, s in enumerate(cfg.workers) if s.kind == st.DQSG and s.bits == 2 and (s.levels or 3) == 3]
+    if tern:
+        # three-level messages: the radix-3 container (five codes per byte) and back; only packed data is touched
+        src = [m[tern[0]].packed for m in msg_sets]
+        data = [dq.ternary_pack(p_, n) for p_ in src]
+        by_t = 4 * dq.packed_words(n, 2) + dq.ternary_bytes(n)
+        ms_p = time_isolated(torch, [(lambda a=src[i], b=data[i]: dq.ternary_pack(a, n, b)) for i in range(sets)])
+        ms_u = time_isolated(torch, [(lambda a=data[i], b=src[i]: dq.ternary_unpack(a, n, b)) for i in range(sets)])
+        for name, ms_t in (("ternary_pack", ms_p), ("ternary_unpack", ms_u)):
+            res[name] = {"ms": ms_t, "bytes": by_t, "gbs": by_t / ms_t / 1e6, "gelem_s": n / ms_t / 1e6,
+                         "frac_hbm": by_t / ms_t / 1e6 / hbm_peak,
+                         "container_bits_per_element": 8 * dq.ternary_bytes(n) / n}
     elem_workers = n * cfg.W
     alg_instr = DEC_INSTR_PER_ELEM_WORKER * elem_workers + DEC_INSTR_PER_ELEM * n
     res["decode_aggregate"] = {"ms": ms, "bytes": per_set, "gbs": per_set / ms / 1e6, "gelem_s": n / ms / 1e6,

@@ -54,6 +54,8 @@ typedef enum { DQ_KIND_DQSG = 0, DQ_KIND_NDQSG = 1 } dq_kind;
 #define DQ_WARN_NONFINITE_SCALE 0x1u   /* a received scale was NaN or Inf                                   */
 #define DQ_ERR_COPY_TIMEOUT     0x2u   /* a bounded wait for an asynchronous tile copy ran out; the tile
                                           was skipped and its outputs are undefined                        */
+#define DQ_WARN_CODE_RANGE      0x4u   /* dq_ternary_pack met a code 3 (not a three-level message); it was
+                                          stored as 2                                                      */
 
 /* One quantizer description.  Plain data, read during the call. */
 typedef struct {
@@ -160,6 +162,27 @@ dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_
  *   hist    device, uint64[2^bits], 8-byte aligned; zeroed and filled by the call
  */
 dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, uint64_t* hist, void* cuda_stream);
+
+/*
+ * Radix-3 container for three-level DQSG messages (levels = 3, bits = 2).  Section 4 counts log2(3) = 1.585
+ * bits per element for the three-level quantizer (raw-bits table, DQSGD row); the 2-bit stream spends 2.  The
+ * container stores five codes per byte,
+ *     byte k = t_{5k} + 3 t_{5k+1} + 9 t_{5k+2} + 27 t_{5k+3} + 81 t_{5k+4}   (codes past n count as 0),
+ * i.e. 1.6 bits per element: 20 % fewer bytes on the wire, within 1 % of the paper's count.  The scales are
+ * sent unchanged.  The encode and decode-aggregate kernels keep working on the 2-bit stream; these two calls
+ * convert a message between the two forms on the device and touch only the packed data.
+ *   dq_ternary_bytes   ceil(n / 5), the size of the container
+ *   dq_ternary_pack    packed: device, dq_packed_words(n, 2) words whose codes are 0, 1 or 2 (a code 3 is
+ *                      stored as 2 and DQ_WARN_CODE_RANGE is OR-ed into *status_word when that is not NULL);
+ *                      out_radix: device, dq_ternary_bytes(n) bytes, 16-byte aligned, fully overwritten
+ *   dq_ternary_unpack  radix: device, dq_ternary_bytes(n) bytes (a byte above 242 is read as its five
+ *                      low base-3 digits); out_packed: device, dq_packed_words(n, 2) words, fully
+ *                      overwritten, pad bits 0 -- bit-identical to the stream that was packed
+ */
+uint64_t dq_ternary_bytes(uint64_t n);
+dq_status dq_ternary_pack(const uint32_t* packed, uint64_t n, uint8_t* out_radix, uint32_t* status_word,
+                          void* cuda_stream);
+dq_status dq_ternary_unpack(const uint8_t* radix, uint64_t n, uint32_t* out_packed, void* cuda_stream);
 
 /*
  * Host-buffer variants.  Every data pointer (grad, out_packed, out_scale, the packed/scale pointers

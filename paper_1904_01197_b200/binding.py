@@ -17,6 +17,7 @@ DQ_KIND_DQSG = 0
 DQ_KIND_NDQSG = 1
 DQ_WARN_NONFINITE_SCALE = 0x1
 DQ_ERR_COPY_TIMEOUT = 0x2
+DQ_WARN_CODE_RANGE = 0x4
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libdq_b200.so"
 
@@ -68,6 +69,9 @@ def lib() -> C.CDLL:
         L.ndqsg_decode_aggregate_running.restype = C.c_int
         L.dq_code_histogram.argtypes = [vp, u64, u32, vp, vp]
         L.dq_code_histogram.restype = C.c_int
+        L.dq_ternary_bytes.argtypes = [u64]; L.dq_ternary_bytes.restype = u64
+        L.dq_ternary_pack.argtypes = [vp, u64, vp, vp, vp]; L.dq_ternary_pack.restype = C.c_int
+        L.dq_ternary_unpack.argtypes = [vp, u64, vp, vp]; L.dq_ternary_unpack.restype = C.c_int
         L.dq_encode_workspace_bytes.argtypes = [u64, pp]; L.dq_encode_workspace_bytes.restype = u64
         L.dq_decode_workspace_bytes.argtypes = [pm, u32, u64, C.c_int]; L.dq_decode_workspace_bytes.restype = u64
         for f in (L.dqsg_encode_host, L.ndqsg_encode_host):
@@ -251,6 +255,31 @@ def entropy_bits_per_element(hist) -> float:
     counts = [int(c) for c in hist.tolist()]
     total = sum(counts)
     return -sum(c / total * math.log2(c / total) for c in counts if c) if total else 0.0
+
+
+# ------------------------------------------------------------------------------------------ radix-3 container
+def ternary_bytes(n: int) -> int:
+    return int(lib().dq_ternary_bytes(n))
+
+
+def ternary_pack(packed: torch.Tensor, n: int, out: Optional[torch.Tensor] = None,
+                 status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """2-bit stream of a three-level message -> five codes per byte (uint8[ternary_bytes(n)] on the device)."""
+    if out is None:
+        out = torch.empty(max(1, ternary_bytes(n)), dtype=torch.uint8, device=packed.device)
+    _check(lib().dq_ternary_pack(_dev_ptr(packed, torch.int32, "packed"), n, _dev_ptr(out, torch.uint8, "out"),
+                                 _dev_ptr(status_word, torch.int32, "status_word"), _stream_ptr(stream)),
+           "dq_ternary_pack")
+    return out
+
+
+def ternary_unpack(data: torch.Tensor, n: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Five codes per byte -> the 2-bit stream (int32[packed_words(n, 2)] on the device)."""
+    if out is None:
+        out = torch.empty(max(1, packed_words(n, 2)), dtype=torch.int32, device=data.device)
+    _check(lib().dq_ternary_unpack(_dev_ptr(data, torch.uint8, "data"), n, _dev_ptr(out, torch.int32, "out"),
+                                   _stream_ptr(stream)), "dq_ternary_unpack")
+    return out
 
 
 # ------------------------------------------------------------------------------------------ host buffers

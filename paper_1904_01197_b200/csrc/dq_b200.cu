@@ -10,6 +10,7 @@
 #include "dq_decode.cuh"
 #include "dq_encode.cuh"
 #include "dq_stats.cuh"
+#include "dq_ternary.cuh"
 
 namespace {
 
@@ -423,6 +424,42 @@ dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, u
     static_assert(sizeof(unsigned long long) == sizeof(uint64_t), "histogram counters are 64-bit");
     if (launch_overlapped(dq::code_histogram_kernel, (uint32_t)grid, (uint32_t)dq::kHistThreads, 0, st, packed, n,
                           bits, reinterpret_cast<unsigned long long*>(hist)) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return DQ_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ radix-3 container
+uint64_t dq_ternary_bytes(uint64_t n) { return (n + 4u) / 5u; }
+
+static_assert(dq::kWarnCodeRange == DQ_WARN_CODE_RANGE, "status bit of the container kernels");
+
+dq_status dq_ternary_pack(const uint32_t* packed, uint64_t n, uint8_t* out_radix, uint32_t* status_word,
+                          void* cuda_stream)
+{
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    if (n == 0) return DQ_OK;
+    if (!packed || !out_radix) return DQ_ERR_INVALID_ARG;
+    if (!aligned16(packed) || !aligned16(out_radix)) return DQ_ERR_ALIGNMENT;
+    const uint64_t units = (n + 79u) / 80u;
+    const uint64_t grid = (units + dq::kTernaryThreads - 1u) / dq::kTernaryThreads;
+    if (launch_overlapped(dq::ternary_pack_kernel, (uint32_t)grid, (uint32_t)dq::kTernaryThreads, 0,
+                          static_cast<cudaStream_t>(cuda_stream), packed, n, out_radix, status_word) != cudaSuccess)
+        return DQ_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return DQ_OK;
+}
+
+dq_status dq_ternary_unpack(const uint8_t* radix, uint64_t n, uint32_t* out_packed, void* cuda_stream)
+{
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    if (n == 0) return DQ_OK;
+    if (!radix || !out_packed) return DQ_ERR_INVALID_ARG;
+    if (!aligned16(radix) || !aligned16(out_packed)) return DQ_ERR_ALIGNMENT;
+    const uint64_t units = (n + 79u) / 80u;
+    const uint64_t grid = (units + dq::kTernaryThreads - 1u) / dq::kTernaryThreads;
+    if (launch_overlapped(dq::ternary_unpack_kernel, (uint32_t)grid, (uint32_t)dq::kTernaryThreads, 0,
+                          static_cast<cudaStream_t>(cuda_stream), radix, n, out_packed) != cudaSuccess)
         return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;
