@@ -214,6 +214,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     // in the same launch
     const int sms = device_sm_count();
     if (sms <= 0) return DQ_ERR_CUDA;
+    a.sm_count = (uint32_t)sms;
     const uint32_t B = p->bucket;
     const uint32_t U = (B < 1024u) ? 1024u : B;                     // elements per work unit
     uint64_t tiles = (is_pow2(B) && B <= 8192u) ? n / U : 0u;       // whole units
@@ -250,6 +251,8 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
         const uint64_t want_ctas = (tiles + groups_per_cta - 1u) / groups_per_cta;
         tile_ctas = (uint32_t)(want_ctas < room ? want_ctas : room);
     }
+    // the spacing only pays when the first requests of all resident warps saturate HBM
+    a.request_spacing_ns = (uint32_t)((uint64_t)dq::kFirstRequestSpacingNs * tile_ctas / slots);
     cudaError_t e;
     const bool d16 = (p->dither_bits == 16u);
     if (mode == dq::kEncDqsg) e = launch_encode<dq::kEncDqsg>(p->bits, d16, map, a, plain + tile_ctas, st);

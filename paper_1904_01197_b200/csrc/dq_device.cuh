@@ -203,6 +203,13 @@ __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
 // Programmatic dependent launch: wait until the previous kernel of the stream has completed and its writes are
 // visible (a no-op when the kernel was launched normally), and allow the next kernel to begin launching.
 __device__ __forceinline__ void grid_dependency_wait()

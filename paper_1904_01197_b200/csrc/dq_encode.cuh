@@ -37,6 +37,8 @@ constexpr int kEncThreads = 32 * kConsumerWarps;
 constexpr int kEncStages = DQ_ENC_STAGES;
 constexpr int kEncCtasPerSm = DQ_ENC_CTAS_PER_SM;
 constexpr size_t kEncSmemBytes = (size_t)kEncStages * kTileBytes + 1024;
+// Time HBM needs to deliver one warp's pipeline stages (8 KB) to each of the 148 SMs: 148 x 8 KB / 6.5 TB/s.
+constexpr uint32_t kFirstRequestSpacingNs = 190u;
 
 struct EncodeArgs {
     const float* grad;
@@ -58,6 +60,8 @@ struct EncodeArgs {
     float kmax;              // DQSG: L - 1
     uint32_t K;              // NDQSG: coarse ratio
     uint32_t K_offset;       // NDQSG any K: multiple of K that is >= 2^22
+    uint32_t sm_count;       // SMs of the device            } spacing of the first tile requests,
+    uint32_t request_spacing_ns;   // see encode_kernel      } 0 when the grid does not fill the device
     PhiloxStream ps;
 };
 
@@ -290,6 +294,14 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     // nothing above touches memory that an earlier kernel of the stream may still be writing
     grid_dependency_wait();
     if (lane == 0) {
+        // All resident warps would request their first tiles (the whole shared memory of every SM, a quarter of a
+        // ResNet-50-sized gradient) at the same instant; served interleaved, every warp would then get its data
+        // late and the ALUs would idle for 3-6 us.  Spacing the requests of an SM's warps at the rate at which
+        // HBM can serve them lets the first warps start after about 1 us while the memory system stays busy.
+        // (CTAs are assumed to be placed round-robin over the SMs; any other placement only changes the order.)
+        const uint32_t rank = ((blockIdx.x - args.plain_ctas) / args.sm_count) * (uint32_t)kConsumerWarps + warp;
+        const uint64_t until = global_timer_ns() + (uint64_t)rank * args.request_spacing_ns;
+        for (uint32_t it = 0; it < 4096u && args.request_spacing_ns != 0u && global_timer_ns() < until; ++it) { }
 #pragma unroll
         for (int s = 0; s < kEncStages; ++s) {
             // first copies: the next two units of this warp, or (pair mode) the two halves of its first bucket
