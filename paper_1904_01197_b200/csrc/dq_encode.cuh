@@ -299,6 +299,8 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         // late and the ALUs would idle for 3-6 us.  Spacing the requests of an SM's warps at the rate at which
         // HBM can serve them lets the first warps start after about 1 us while the memory system stays busy.
         // (CTAs are assumed to be placed round-robin over the SMs; any other placement only changes the order.)
+        // The CTAs with the lowest indices go first; they are also the ones whose warps take one unit more when
+        // the units do not divide evenly, so the longest-running warps start earliest.
         const uint32_t rank = ((blockIdx.x - args.plain_ctas) / args.sm_count) * (uint32_t)kConsumerWarps + warp;
         const uint64_t until = global_timer_ns() + (uint64_t)rank * args.request_spacing_ns;
         for (uint32_t it = 0; it < 4096u && args.request_spacing_ns != 0u && global_timer_ns() < until; ++it) { }
