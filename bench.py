@@ -39,17 +39,19 @@ SM_COUNT, ISSUE_PER_SM_CLK, LANES = 148, 4, 32           # ALU-issue ceiling: SM
 # Algorithmic lane-instructions: ~22 per (element, worker) + ~10 per element for the fused decode,
 # ~24 per element for the encode.
 DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 24.0
-# Executed lane-instructions per (element, worker) of the fused decode on the ResNet-50-sized workload, split into
-# the half-rate class (integer, logic, IMAD, shifts, branches, loads) and fp32, from the opcode counters in
-# profiles/decode_aggregate_kernel_ndqsg_resnet50.md: the issue ceiling of that mix is
-# schedulers x lanes x clock / (2 * half_rate + fp32).
-DEC_MIX = {32: (17.0, 8.8), 16: (13.2, 8.8)}
+# Executed lane-instructions per (element, worker) of the fused decode on the ResNet-50-sized workload, from the
+# opcode counters in profiles/decode_aggregate_kernel_ndqsg_resnet50.md: (32x32->64 multiplies, fp32 adds /
+# multiplies / multiply-adds, everything else).  Their scheduler cost is taken from the issue probe
+# (profiles/issue_cost_probe_b200.md): 4.4 cycles per wide multiply with one other instruction hidden behind it,
+# 1 cycle per fp32 instruction, 2 cycles for the rest; the classes add up.
+DEC_MIX = {32: (4.29, 9.82, 12.22), 16: (2.18, 9.82, 9.58)}
+ISSUE_CYCLES_WIDE, ISSUE_CYCLES_FP32, ISSUE_CYCLES_OTHER = 4.4, 1.0, 2.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
 NCU_TRAFFIC = {
-    ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_689_280,    # profiles/encode_kernel_ndqsg_resnet50.md
-    ("encode", "ndqsg_resnet50", 25_557_032, 3): 105_917_696,
-    ("decode", "ndqsg_resnet50", 25_557_032): 219_741_696,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
+    ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_344_960,    # profiles/encode_kernel_ndqsg_resnet50.md
+    ("encode", "ndqsg_resnet50", 25_557_032, 3): 106_753_792,
+    ("decode", "ndqsg_resnet50", 25_557_032): 220_192_768,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
 }
 
 
@@ -588,8 +590,12 @@ def main():
                                "hbm_gbs": kd["gbs"], "frac_hbm": kd["frac_hbm"], "launches_per_step": 1}
             mix = DEC_MIX.get(cfg.workers[0].dither_bits)
             if mix and cfg.name == "ndqsg_resnet50":
-                ceiling = SM_COUNT * ISSUE_PER_SM_CLK * LANES * sm_max_mhz * 1e6 / (2.0 * mix[0] + mix[1])
-                roofline_decode["issue_mix"] = {"half_rate_instr_per_unit": mix[0], "fp32_instr_per_unit": mix[1],
+                wide, fp32, other = mix
+                cycles = (ISSUE_CYCLES_WIDE * wide + ISSUE_CYCLES_FP32 * fp32 +
+                          ISSUE_CYCLES_OTHER * max(0.0, other - wide))
+                ceiling = SM_COUNT * ISSUE_PER_SM_CLK * LANES * sm_max_mhz * 1e6 / cycles
+                roofline_decode["issue_mix"] = {"wide_mul_per_unit": wide, "fp32_instr_per_unit": fp32,
+                                                "other_instr_per_unit": other, "scheduler_cycles_per_unit": cycles,
                                                 "ceiling_gelem_worker_s": ceiling / 1e9,
                                                 "frac_of_ceiling": kd["gelem_worker_s"] * 1e9 / ceiling}
             if kd["ms"] >= count[dom_enc] * ke["ms"]:
