@@ -202,7 +202,10 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
         a.gain_num = a.shift;
         a.kmax = (float)(L - 1u);
     } else {
-        mode = is_pow2(p->coarse_K) ? dq::kEncNdqsgPow2 : dq::kEncNdqsgAnyK;
+        // The power-of-two path keeps the low `bits` bits of the index when bits divides 32 (K = 2^bits) and masks
+        // with K - 1 otherwise; a power of two below 2^bits with such a width takes the general path.
+        const bool low_bits_are_the_coset = (p->coarse_K == (1u << p->bits)) || (32u % p->bits) != 0u;
+        mode = (is_pow2(p->coarse_K) && low_bits_are_the_coset) ? dq::kEncNdqsgPow2 : dq::kEncNdqsgAnyK;
         a.gain_num = alpha * p->fine_M;
         a.K = p->coarse_K;
         a.K_offset = ((4194304u + p->coarse_K - 1u) / p->coarse_K) * p->coarse_K;

@@ -128,6 +128,7 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, f
         for (int j = 0; j < 4; ++j) ctr[j] = row * (32u / EPB) + (uint32_t)(4 * h + j);
         philox4x32_10_xN<4>(ctr, args.ps, rnd);
         if constexpr (MODE == kEncNdqsgPow2 && (32 % BITS) == 0) {
+            // K = 2^BITS here (the host sends any smaller power of two down the general path)
             // units of U elements (a whole word, or half a word for one bit); elements are inserted from the
             // last to the first: moving the code to the top of a register drops the bits above it, and one
             // funnel shift pushes it into the unit.

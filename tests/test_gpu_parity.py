@@ -76,6 +76,19 @@ def test_encode_bit_exact_bucket_sizes(dq, oracle, bucket):
         _check_encode(dq, oracle, g, spec, worker=1, step=9, bucket=bucket)
 
 
+@pytest.mark.parametrize("bits", range(2, 9))
+def test_encode_coarse_ratio_below_the_field_width(dq, oracle, bits):
+    # every power of two K < 2^bits: the code is q1 mod K, not the low `bits` bits of q1
+    rng = np.random.default_rng(250 + bits)
+    n = 3 * 2048 + 8192 + 57
+    g = (rng.standard_normal(n) * 0.3).astype(np.float32)
+    for logk in range(1, bits):
+        spec = WorkerSpec(NDQSG, bits, 0, 1 << logk, float(3 << logk), 1.0, 40 + logk)
+        for bucket in (2048, 96):
+            pk, sc, opk, osc = _check_encode(dq, oracle, g, spec, worker=2, step=5, bucket=bucket)
+        assert oracle.unpack(opk, n, bits).max() < (1 << logk)
+
+
 @pytest.mark.parametrize("n", [1, 3, 31, 32, 33, 100, 1023, 1024, 1025, 2048, 4097, 8191])
 def test_encode_ragged_lengths(dq, oracle, n):
     rng = np.random.default_rng(300 + n)
