@@ -29,7 +29,7 @@ def _random_spec(rng, dither_bits):
     return WorkerSpec(NDQSG, bits, 0, K, M1, alpha, seed, dither_bits=dither_bits)
 
 
-@pytest.mark.parametrize("case", range(24))
+@pytest.mark.parametrize("case", range(48))
 def test_random_configuration(dq, oracle, case):
     rng = np.random.default_rng(77_000 + case)
     bucket = int(rng.choice(BUCKETS))
@@ -46,4 +46,57 @@ def test_random_configuration(dq, oracle, case):
         _check_encode(dq, oracle, grads[w], specs[w], worker=w, step=step, bucket=bucket)
     got, ref = _roundtrip_decode(dq, oracle, W, n, bucket, specs, grads, side, step)
     assert_fp32_close(got, ref, f"case {case}: bucket={bucket} n={n} W={W} specs={specs}")
+    assert dq.device_error_flags() == 0
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_random_running_mean_configuration(dq, oracle, case):
+    # Algorithm 2's server loop: the first message is DQSG, the rest are drawn at random
+    from test_gpu_running_mean import _run
+    rng = np.random.default_rng(78_000 + case)
+    bucket = int(rng.choice(BUCKETS))
+    n = int(rng.integers(1, 6)) * bucket + int(rng.integers(0, bucket)) + (0 if case % 3 else 8192 * 2)
+    W = int(rng.integers(2, 7))
+    dither_bits = 16 if case % 2 else 32
+    step = int(rng.integers(0, 2 ** 40))
+    c = rng.standard_normal(n).astype(np.float32)
+    grads = [(c + 0.2 * rng.standard_normal(n)).astype(np.float32) for _ in range(W)]
+    first = WorkerSpec(DQSG, 3, int(rng.integers(2, 9)), seed=int(rng.integers(0, 2 ** 63)), dither_bits=dither_bits)
+    specs = [first] + [_random_spec(rng, dither_bits) for _ in range(W - 1)]
+    got, ref = _run(dq, oracle, specs, grads, n, bucket, step)
+    assert_fp32_close(got, ref, f"case {case}: bucket={bucket} n={n} specs={specs}")
+
+
+@pytest.mark.parametrize("case", range(6))
+def test_random_host_buffer_round_trip(dq, oracle, case):
+    # the host-buffer entry points on random configurations: same bits and the same mean as the oracle
+    from dq_testlib import oracle_encode, oracle_msg, spec_params
+    rng = np.random.default_rng(79_000 + case)
+    bucket = int(rng.choice(BUCKETS))
+    n = int(rng.integers(1, 6)) * bucket + int(rng.integers(0, bucket))
+    W = int(rng.integers(1, 5))
+    dither_bits = 16 if case % 2 else 32
+    step = int(rng.integers(0, 2 ** 40))
+    side = rng.standard_normal(n).astype(np.float32)
+    grads = [(side + 0.1 * rng.standard_normal(n)).astype(np.float32) for _ in range(W)]
+    specs = [_random_spec(rng, dither_bits) for _ in range(W)]
+    host_msgs, omsgs = [], []
+    for w, (g, sp) in enumerate(zip(grads, specs)):
+        p = spec_params(dq, sp, bucket)
+        pk = torch.empty(max(1, dq.packed_words(n, sp.bits)), dtype=torch.int32).pin_memory()
+        sc = torch.empty(max(1, dq.num_buckets(n, bucket)), dtype=torch.float32).pin_memory()
+        ws = torch.empty(dq.encode_workspace_bytes(n, p), dtype=torch.uint8, device="cuda")
+        fn = dq.dqsg_encode_host if sp.kind == DQSG else dq.ndqsg_encode_host
+        fn(torch.from_numpy(g).pin_memory(), sp.seed, w, step, p, pk, sc, ws)
+        opk, osc = oracle_encode(oracle, g, sp, w, step, bucket)
+        assert np.array_equal(pk.numpy().view(np.uint32)[:opk.size], opk), f"case {case}: worker {w} {sp}"
+        assert np.array_equal(sc.numpy()[:osc.size].view(np.uint32), osc.view(np.uint32))
+        host_msgs.append(dq.Message(pk, sc, sp.seed, w, sp.kind, p))
+        omsgs.append(oracle_msg(oracle, opk, osc, sp, w, bucket))
+    any_nd = any(s.kind == NDQSG for s in specs)
+    out = torch.empty(n, dtype=torch.float32).pin_memory()
+    ws = torch.empty(dq.decode_workspace_bytes(host_msgs, n, any_nd), dtype=torch.uint8, device="cuda")
+    dq.ndqsg_decode_aggregate_host(host_msgs, n, step, torch.from_numpy(side).pin_memory() if any_nd else None, out, ws)
+    ref = oracle.decode_aggregate(omsgs, n, step, side_info=side if any_nd else None, threads=4)
+    assert_fp32_close(out.numpy(), ref, f"case {case}")
     assert dq.device_error_flags() == 0
