@@ -224,8 +224,8 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     if (tiles > 0xFFFFFFFFull) return DQ_ERR_UNSUPPORTED;
     CUtensorMap map;
     std::memset(&map, 0, sizeof(map));
-    const bool pair = (B == 2048u);                                 // one warp per 2048-bucket, two halves in time
-    const uint32_t wpb = (B < 1024u || pair) ? 1u : (B / 1024u);
+    const bool pair = (B == 2048u || B == 4096u || B == 8192u);     // a warp takes 2048 elements, two halves in time
+    const uint32_t wpb = pair ? (B / 2048u) : (B < 1024u) ? 1u : (B / 1024u);
     a.pair_in_time = pair ? 1u : 0u;
     if (tiles > 0) {
         if (!make_row_map(&map, grad, tiles * (U / 32u), 32u)) return DQ_ERR_CUDA;

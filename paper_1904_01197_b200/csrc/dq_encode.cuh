@@ -5,13 +5,17 @@
 // `bits` 32-bit words of the bit stream.  One lane quantizes and packs a whole row, so no lane ever shares a
 // packed word with another lane and no shuffles are needed for packing.
 //
-// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight warps.  The warps of a CTA form
-// groups of B/1024 warps (one warp for smaller buckets); the groups of all CTAs take work units -- one bucket,
-// or 1024 elements -- round-robin.  Every warp owns 32 rows of each unit and keeps its own two-stage
-// shared-memory pipeline filled with asynchronous 2-D tile copies (128-byte swizzle, which makes "lane r reads
-// row r" free of bank conflicts): it takes its rows of a stage into registers, re-arms the stage with the copy
-// for the unit after next, reduces max|g| over its bucket (shuffles inside the warp, a named barrier between
-// the warps that share a bucket) and then quantizes from registers.  The gradient is read from HBM exactly once.
+// Power-of-two buckets up to 8192 take the tile path: persistent CTAs of eight warps, every warp with its own
+// two-stage shared-memory pipeline of 4 KB tiles (32 rows) filled by asynchronous 2-D tile copies (128-byte
+// swizzle, which makes "lane r reads row r" free of bank conflicts).
+//   B <= 1024: a work unit is 1024 elements; a warp takes a stage into registers, re-arms the stage with the
+//     copy for the unit after next, reduces max|g| over each bucket with shuffles and quantizes from registers.
+//   B = 2048, 4096, 8192: a work unit is a bucket and a warp takes 2048 elements of it as two halves in time,
+//     one per stage: when both have landed it reads the maximum of the second half from shared memory, takes the
+//     first half into registers, and quantizes one half after the other, re-arming each stage as soon as it is
+//     in registers.  For B = 2048 no other warp is involved; for 4096 and 8192 the two or four warps of a bucket
+//     meet once per bucket in a named barrier to exchange their maxima.
+// The units are dealt out round-robin over the warp groups of all CTAs.  The gradient is read from HBM exactly once.
 //
 // Everything else -- other bucket sizes, the part of the vector past the last whole tile, the ragged end --
 // is handled by plain-load code, one warp per bucket, in extra CTAs of the same launch.
@@ -53,8 +57,9 @@ struct EncodeArgs {
     uint32_t bucket;         // B
     uint32_t bucket_log2;    // log2(B) on the tile path
     uint32_t lanes_per_bucket;  // B / 32 when B < 1024, else 32
-    uint32_t warps_per_bucket;  // B / 1024 when B >= 1024, else 1
-    uint32_t pair_in_time;      // B == 2048: one warp handles both halves of a bucket (units are buckets)
+    uint32_t warps_per_bucket;  // B / 2048 when B >= 2048, else 1
+    uint32_t pair_in_time;      // B = 2048, 4096, 8192: a warp handles 2048 elements of a bucket as two halves in
+                                // time; warps_per_bucket = B / 2048 warps share a bucket (units are buckets)
     float gain_num;          // DQSG: s = (L-1)/2;  NDQSG: A = alpha * M1
     float shift;             // DQSG: s
     float kmax;              // DQSG: L - 1
@@ -245,10 +250,9 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
 // The encode kernel.  Grid = CTAs for the plain-load part (scheduled first) + persistent tile CTAs.
 // Block = 8 warps.  Dynamic shared memory = kEncSmemBytes.
 //
-// Tile path: the warps of a CTA form groups (one group per bucket position); a group walks over work units
-// and each of its warps owns 32 rows of every unit and runs its own two-stage pipeline: its lane 0 issues the 4 KB tile copy for the tile after next as soon as
-// the warp has taken the current rows into registers, so a copy is always in flight while the warp
-// quantizes, and no warp ever waits for another one except the warps that share a bucket (named barrier).
+// Tile path: lane 0 of every warp issues the 4 KB tile copy for its next unit as soon as the warp has taken the
+// current rows into registers, so a copy is always in flight while the warp quantizes, and no warp ever waits
+// for another one except the warps that share a bucket of 4096 or 8192 elements (named barrier, once per bucket).
 // ---------------------------------------------------------------------------------------------------
 template <int BITS, int MODE, int DITH>
 __global__ void __launch_bounds__(kEncThreads, kEncCtasPerSm)
@@ -275,16 +279,14 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t my_smem = smem_base + warp * (uint32_t)(kEncStages * kWarpTileBytes);
     const uint32_t my_bar = smem_u32(&bar_full[warp][0]);
-    // Work unit = the rows of one bucket (B >= 1024: B / 1024 warps work on it together) or 1024 elements
-    // (smaller buckets: one warp).  The groups of all tile CTAs take units round-robin, which spreads the work
-    // over the SMs to within one unit.
-    const uint32_t wpb = args.warps_per_bucket;      // warps sharing a bucket (1, 2, 4, 8)
+    // Work unit = one bucket (B >= 2048: B / 2048 warps work on it together) or 1024 elements (smaller buckets:
+    // one warp).  The groups of all tile CTAs take units round-robin, which spreads the work over the SMs to
+    // within one unit.
+    const uint32_t wpb = args.warps_per_bucket;      // warps sharing a bucket (1, 2, 4)
     const uint32_t group = warp / wpb;               // group of this warp inside the CTA
     const uint32_t groups_per_cta = (uint32_t)kConsumerWarps / wpb;
     const uint32_t stride = (gridDim.x - args.plain_ctas) * groups_per_cta;
     const uint32_t first_tile = (blockIdx.x - args.plain_ctas) * groups_per_cta + group;
-    const uint32_t unit_rows = wpb * 32u;
-    const uint32_t row_in_unit = (warp % wpb) * 32u;
 
     if (lane == 0) {
 #pragma unroll
@@ -309,7 +311,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         for (int s = 0; s < kEncStages; ++s) {
             // first copies: the next two units of this warp, or (pair mode) the two halves of its first bucket
             const uint64_t tile = args.pair_in_time ? (uint64_t)first_tile : (uint64_t)first_tile + (uint64_t)s * stride;
-            const uint64_t row0 = args.pair_in_time ? tile * 64u + (uint64_t)s * 32u : tile * unit_rows + row_in_unit;
+            const uint64_t row0 = args.pair_in_time ? (tile * wpb + warp % wpb) * 64u + (uint64_t)s * 32u : tile * 32u;
             if (tile < args.num_units) {
                 mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
                 tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s, (int32_t)row0);
@@ -326,8 +328,12 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         // B = 2048: one warp handles the whole bucket as two consecutive 1024-element halves, one per stage, so
         // no other warp is involved.  The second half only has to have landed (it was requested a whole unit
         // earlier) for its maximum to be read from shared memory before the first half is quantized.
+        // B = 4096, 8192: the same, with two or four warps taking 2048 elements each and meeting once per bucket
+        // to exchange their maxima.
+        const uint32_t sub = warp % wpb;                 // this warp's 2048-element part of the bucket
         for (uint64_t pair = first_tile; pair < args.num_units; pair += stride, ++k) {
             const uint32_t par = k & 1u;
+            const uint64_t part = pair * wpb + sub;      // index of this warp's 2048 elements in the gradient
             float x[32];
             float mx = 0.0f;
 #pragma unroll 1
@@ -363,7 +369,16 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                     for (int e = 0; e < 32; e += 2) mx = max3_abs(mx, x[e], x[e + 1]);
 #pragma unroll
                     for (uint32_t off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-                    if (lane == 0) args.scale[pair] = mx;
+                    if (wpb > 1u) {
+                        if (lane == 0) warp_max[par][warp] = mx;
+                        named_bar_sync(1u + group, wpb * 32u);
+#pragma unroll
+                        for (uint32_t i = 0; i < (uint32_t)kConsumerWarps; ++i) {
+                            const float o = warp_max[par][i];
+                            if (i / wpb == group) mx = fmaxf(mx, o);
+                        }
+                    }
+                    if (lane == 0 && sub == 0u) args.scale[pair] = mx;
                 } else {
                     uint32_t sink = 0u;                 // all loads of this half have completed after this
 #pragma unroll
@@ -376,11 +391,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                     if (next < args.num_units) {
                         mbar_expect_tx(my_bar + 8u * half, (uint32_t)kWarpTileBytes);
                         tma_load_rows(my_smem + half * kWarpTileBytes, &tmap, my_bar + 8u * half,
-                                      (int32_t)(next * 64u + half * 32u));
+                                      (int32_t)((next * wpb + sub) * 64u + half * 32u));
                     }
                 }
                 const float a = bucket_gain(args.gain_num, mx);
-                const uint32_t row = (uint32_t)pair * 64u + half * 32u + lane;
+                const uint32_t row = (uint32_t)part * 64u + half * 32u + lane;
                 uint32_t out[BITS];
                 encode_row<BITS, MODE, DITH>(x, row, a, args, out);
                 store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
@@ -389,6 +404,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         return;
     }
 
+    // buckets of 1024 elements or fewer: a unit is 1024 elements, one warp, one row per lane
     for (uint64_t tile = first_tile; tile < args.num_units; tile += stride, ++k) {
         const uint32_t s = k % kEncStages;
         const uint32_t use = k / kEncStages;
@@ -422,23 +438,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
             if (next < args.num_units) {
                 mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
                 tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
-                              (int32_t)(next * unit_rows + row_in_unit));
+                              (int32_t)(next * 32u));
             }
         }
-        const uint32_t row = (uint32_t)tile * unit_rows + row_in_unit + lane;   // row index in the gradient (< 2^29)
-        if (wpb > 1u) {
-            if (lane == 0) warp_max[k & 1u][warp] = mx;
-            named_bar_sync(1u + group, wpb * 32u);
-            // the maximum over the bucket's warps: all eight slots are read, the ones of other buckets ignored
-#pragma unroll
-            for (uint32_t i = 0; i < (uint32_t)kConsumerWarps; ++i) {
-                const float o = warp_max[k & 1u][i];
-                if (i / wpb == group) mx = fmaxf(mx, o);
-            }
-            if (lane == 0 && (warp % wpb) == 0u) args.scale[row >> (args.bucket_log2 - 5u)] = mx;
-        } else if ((lane & (args.lanes_per_bucket - 1u)) == 0u) {
-            args.scale[row >> (args.bucket_log2 - 5u)] = mx;
-        }
+        const uint32_t row = (uint32_t)tile * 32u + lane;   // row index in the gradient (< 2^29)
+        if ((lane & (args.lanes_per_bucket - 1u)) == 0u) args.scale[row >> (args.bucket_log2 - 5u)] = mx;
         const float a = bucket_gain(args.gain_num, mx);
 
         uint32_t out[BITS];
