@@ -155,6 +155,33 @@ dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_
                                          float* out_avg, uint32_t* status_word, void* cuda_stream);
 
 /*
+ * Bucket ranges.  Buckets are independent and the dither of an element depends on its index in the whole
+ * gradient only (Algorithm 1: every worker quantizes its own coordinates with its own seed; partitioning
+ * paragraph of Section 3.1: one scale per partition), so a gradient can be encoded and decoded in pieces: by
+ * layer as the backward pass produces them, in chunks that overlap with a transfer, or one bucket range per GPU.
+ * The *_range calls work on the elements [first_element, first_element + n) of a longer vector:
+ *   first_element   index of the first element in the whole gradient; a multiple of p->bucket (of the messages'
+ *                   bucket size for the decoder), else DQ_ERR_INVALID_ARG; first_element + n < 2^34
+ *   grad, side_info, out_avg, out_packed, out_scale and the packed / scale pointers inside msgs
+ *                   point at the RANGE's data (element first_element is at index 0), sized for n elements
+ * Because a range starts at a bucket boundary it starts at a word boundary of the bit stream: the messages of
+ * consecutive ranges, concatenated, are bit-identical to the message of one call over the whole vector, and the
+ * decoded ranges are the corresponding slices of the whole result.  first_element = 0 is the plain call.
+ * Every pointer must still be 16-byte aligned: a range may write straight into its slice of whole-gradient
+ * buffers only where that slice is so aligned (first_element * bits a multiple of 128 for the bit stream,
+ * first_element / bucket a multiple of 4 for the scales); otherwise give it buffers of its own.
+ */
+dq_status dqsg_encode_range(const float* grad, uint64_t n, uint64_t first_element, uint64_t seed, uint32_t worker,
+                            uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
+                            void* cuda_stream);
+dq_status ndqsg_encode_range(const float* grad, uint64_t n, uint64_t first_element, uint64_t seed, uint32_t worker,
+                             uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
+                             void* cuda_stream);
+dq_status ndqsg_decode_aggregate_range(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t first_element,
+                                       uint64_t step, const float* side_info, float* out_avg,
+                                       uint32_t* status_word, void* cuda_stream);
+
+/*
  * dq_code_histogram -- counts how often each code occurs in a packed message: hist[c] = number of elements
  * whose b-bit code is c.  This is the input of the paper's rate accounting (Section 4: raw bits are
  * log2(levels) per element, the entropy of the index stream is what an entropy coder approaches).

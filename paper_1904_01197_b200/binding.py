@@ -69,6 +69,10 @@ def lib() -> C.CDLL:
         L.ndqsg_decode_aggregate_running.restype = C.c_int
         L.dq_code_histogram.argtypes = [vp, u64, u32, vp, vp]
         L.dq_code_histogram.restype = C.c_int
+        for f in (L.dqsg_encode_range, L.ndqsg_encode_range):
+            f.argtypes = [vp, u64, u64, u64, u32, u64, pp, vp, vp, vp]; f.restype = C.c_int
+        L.ndqsg_decode_aggregate_range.argtypes = [pm, u32, u64, u64, u64, vp, vp, vp, vp]
+        L.ndqsg_decode_aggregate_range.restype = C.c_int
         L.dq_ternary_bytes.argtypes = [u64]; L.dq_ternary_bytes.restype = u64
         L.dq_ternary_pack.argtypes = [vp, u64, vp, vp, vp]; L.dq_ternary_pack.restype = C.c_int
         L.dq_ternary_unpack.argtypes = [vp, u64, vp, vp]; L.dq_ternary_unpack.restype = C.c_int
@@ -185,6 +189,33 @@ def ndqsg_encode(grad: torch.Tensor, seed: int, worker: int, step: int, params: 
     return _encode(lib().ndqsg_encode, "ndqsg_encode", grad, seed, worker, step, params, out_packed, out_scale, stream)
 
 
+def _encode_range(fn, what, grad, first_element, seed, worker, step, params, out_packed, out_scale, stream):
+    n = grad.numel()
+    if out_packed is None or out_scale is None:
+        out_packed, out_scale = alloc_message(n, params, grad.device)
+    if out_packed.numel() < packed_words(n, params.bits) or out_scale.numel() < num_buckets(n, params.bucket):
+        raise ValueError(f"{what}: output buffers too small")
+    _check(fn(_dev_ptr(grad, torch.float32, "grad"), n, first_element, seed, worker, step, C.byref(params),
+              _dev_ptr(out_packed, torch.int32, "out_packed"), _dev_ptr(out_scale, torch.float32, "out_scale"),
+              _stream_ptr(stream)), what)
+    return out_packed, out_scale
+
+
+def dqsg_encode_range(grad: torch.Tensor, first_element: int, seed: int, worker: int, step: int, params: DqParams,
+                      out_packed: Optional[torch.Tensor] = None, out_scale: Optional[torch.Tensor] = None,
+                      stream=None):
+    """DQSG encode of the elements [first_element, first_element + grad.numel()) of a longer gradient."""
+    return _encode_range(lib().dqsg_encode_range, "dqsg_encode_range", grad, first_element, seed, worker, step,
+                         params, out_packed, out_scale, stream)
+
+
+def ndqsg_encode_range(grad: torch.Tensor, first_element: int, seed: int, worker: int, step: int, params: DqParams,
+                       out_packed: Optional[torch.Tensor] = None, out_scale: Optional[torch.Tensor] = None,
+                       stream=None):
+    return _encode_range(lib().ndqsg_encode_range, "ndqsg_encode_range", grad, first_element, seed, worker, step,
+                         params, out_packed, out_scale, stream)
+
+
 def _msg_array(msgs: Sequence[Message], host: bool = False):
     arr = (DqMsg * max(1, len(msgs)))()
     for i, m in enumerate(msgs):
@@ -212,6 +243,20 @@ def ndqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, side_info
                                         _dev_ptr(out_avg, torch.float32, "out_avg"),
                                         _dev_ptr(status_word, torch.int32, "status_word"), _stream_ptr(stream)),
            "ndqsg_decode_aggregate")
+    return out_avg
+
+
+def ndqsg_decode_aggregate_range(msgs: Sequence[Message], n: int, first_element: int, step: int,
+                                 side_info: Optional[torch.Tensor], out_avg: Optional[torch.Tensor] = None,
+                                 status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Fused decode-and-average of a bucket range: every buffer holds the range's data only."""
+    if out_avg is None:
+        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+    _check(lib().ndqsg_decode_aggregate_range(_msg_array(msgs), len(msgs), n, first_element, step,
+                                              _dev_ptr(side_info, torch.float32, "side_info"),
+                                              _dev_ptr(out_avg, torch.float32, "out_avg"),
+                                              _dev_ptr(status_word, torch.int32, "status_word"),
+                                              _stream_ptr(stream)), "ndqsg_decode_aggregate_range")
     return out_avg
 
 

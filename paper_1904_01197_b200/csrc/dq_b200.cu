@@ -175,14 +175,16 @@ cudaError_t launch_encode(uint32_t bits, bool dither16, const CUtensorMap& map, 
 
 dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t seed, uint32_t worker,
                         uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
-                        cudaStream_t st)
+                        cudaStream_t st, uint64_t first_element = 0u)
 {
     uint32_t L = 0;
     float alpha = 1.0f;
     dq_status s = check_params(p, kind, &L, &alpha);
     if (s != DQ_OK) return s;
+    if (first_element % p->bucket != 0u) return DQ_ERR_INVALID_ARG;      // a range starts at a bucket boundary
     if (n == 0) return DQ_OK;
-    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    if (n >= (1ull << 34) || first_element >= (1ull << 34) || first_element + n >= (1ull << 34))
+        return DQ_ERR_UNSUPPORTED;
     if (!grad || !out_packed || !out_scale) return DQ_ERR_INVALID_ARG;
     if (!aligned16(grad) || !aligned16(out_packed) || !aligned16(out_scale)) return DQ_ERR_ALIGNMENT;
 
@@ -192,6 +194,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     a.packed = out_packed;
     a.scale = out_scale;
     a.n = n;
+    a.row_offset = (uint32_t)(first_element / 32u);
     a.bucket = p->bucket;
     a.num_buckets = dq_num_buckets(n, p->bucket);
     a.num_words = dq_packed_words(n, p->bits);
@@ -268,7 +271,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
 
 dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, const float* side_info,
                         float* out_avg, uint32_t* status_word, bool allow_nested, cudaStream_t st,
-                        bool running = false, bool half_dithered = false)
+                        bool running = false, bool half_dithered = false, uint64_t first_element = 0u)
 {
     if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
     static thread_local dq::DecodeArgs a;    // ~10 KB: keep it off the stack
@@ -310,8 +313,10 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
             }
         }
     }
+    if (first_element % msgs[0].p.bucket != 0u) return DQ_ERR_INVALID_ARG;   // a range starts at a bucket boundary
     if (n == 0) return DQ_OK;
-    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
+    if (n >= (1ull << 34) || first_element >= (1ull << 34) || first_element + n >= (1ull << 34))
+        return DQ_ERR_UNSUPPORTED;
     if (!out_avg) return DQ_ERR_INVALID_ARG;
     if (any_nested && !running && !side_info) return DQ_ERR_INVALID_ARG;
     if (!aligned16(out_avg) || (side_info && !aligned16(side_info))) return DQ_ERR_ALIGNMENT;
@@ -324,6 +329,7 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.status = status_word;
     a.n = n;
     a.rows = (n + 31u) / 32u;
+    a.row_offset = first_element / 32u;
     a.W = W;
     a.rows_per_bucket = msgs[0].p.bucket / 32u;
     a.half_bias_bits = 0x4A800000u;
@@ -410,6 +416,31 @@ dq_status ndqsg_decode_aggregate_running(const dq_msg* msgs, uint32_t W, uint64_
 {
     return decode_common(msgs, W, n, step, nullptr, out_avg, status_word, true,
                          static_cast<cudaStream_t>(cuda_stream), true);
+}
+
+// ------------------------------------------------------------------------------------------------ bucket ranges
+dq_status dqsg_encode_range(const float* grad, uint64_t n, uint64_t first_element, uint64_t seed, uint32_t worker,
+                            uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
+                            void* cuda_stream)
+{
+    return encode_common(DQ_KIND_DQSG, grad, n, seed, worker, step, p, out_packed, out_scale,
+                         static_cast<cudaStream_t>(cuda_stream), first_element);
+}
+
+dq_status ndqsg_encode_range(const float* grad, uint64_t n, uint64_t first_element, uint64_t seed, uint32_t worker,
+                             uint64_t step, const dq_params* p, uint32_t* out_packed, float* out_scale,
+                             void* cuda_stream)
+{
+    return encode_common(DQ_KIND_NDQSG, grad, n, seed, worker, step, p, out_packed, out_scale,
+                         static_cast<cudaStream_t>(cuda_stream), first_element);
+}
+
+dq_status ndqsg_decode_aggregate_range(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t first_element,
+                                       uint64_t step, const float* side_info, float* out_avg,
+                                       uint32_t* status_word, void* cuda_stream)
+{
+    return decode_common(msgs, W, n, step, side_info, out_avg, status_word, true,
+                         static_cast<cudaStream_t>(cuda_stream), false, false, first_element);
 }
 
 dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, uint64_t* hist, void* cuda_stream)

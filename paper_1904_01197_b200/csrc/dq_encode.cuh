@@ -65,6 +65,8 @@ struct EncodeArgs {
     float kmax;              // DQSG: L - 1
     uint32_t K;              // NDQSG: coarse ratio
     uint32_t K_offset;       // NDQSG any K: multiple of K that is >= 2^22
+    uint32_t row_offset;     // index of grad[0]'s row in the whole gradient (0 unless a bucket range is encoded):
+                             // only the dither counters see it
     uint32_t sm_count;       // SMs of the device            } spacing of the first tile requests,
     uint32_t request_spacing_ns;   // see encode_kernel      } 0 when the grid does not fill the device
     PhiloxStream ps;
@@ -108,7 +110,7 @@ __device__ __forceinline__ uint32_t ndqsg_index_bits(float x, float a, float del
 }
 
 // Quantize and pack one row.  x: the 32 elements; row: index of the row in the whole gradient (the Philox
-// counters follow from it); a: the bucket's gain.  out: the row's BITS words.  DITH: 32 or 16 random bits
+// counters follow from it; it differs from the row's position in this call's buffers when a bucket range is encoded); a: the bucket's gain.  out: the row's BITS words.  DITH: 32 or 16 random bits
 // per dither value.
 //
 // Integer and logic instructions cost about twice the issue bandwidth of fp32 ones on this GPU, so the DQSG
@@ -228,7 +230,7 @@ __device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint
         }
         uint32_t out[BITS];
         const uint64_t grow = (lo >> 5) + r;
-        encode_row<BITS, MODE, DITH>(x, (uint32_t)grow, a, args, out);
+        encode_row<BITS, MODE, DITH>(x, (uint32_t)grow + args.row_offset, a, args, out);
         uint32_t* dst = args.packed + grow * BITS;
         if (nvalid == 32u) {
             store_row_words<BITS>(dst, out);
@@ -397,7 +399,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                 const float a = bucket_gain(args.gain_num, mx);
                 const uint32_t row = (uint32_t)part * 64u + half * 32u + lane;
                 uint32_t out[BITS];
-                encode_row<BITS, MODE, DITH>(x, row, a, args, out);
+                encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
                 store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
             }
         }
@@ -446,7 +448,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         const float a = bucket_gain(args.gain_num, mx);
 
         uint32_t out[BITS];
-        encode_row<BITS, MODE, DITH>(x, row, a, args, out);
+        encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
         store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
     }
 }
