@@ -17,6 +17,14 @@ namespace {
 std::atomic<uint64_t> g_launches{0};
 
 bool is_pow2(uint32_t v) { return v && !(v & (v - 1u)); }
+
+// Address of element 0 of the virtual whole-gradient array whose element `first` is p[0] (integer arithmetic: the
+// result may lie outside any allocation and is only ever used with indices >= first).
+template <typename T>
+T* virtual_base(T* p, uint64_t first)
+{
+    return reinterpret_cast<T*>(reinterpret_cast<uintptr_t>(p) - first * sizeof(T));
+}
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0u; }
 
 void fill_philox(dq::PhiloxStream& ps, uint64_t seed, uint32_t worker, uint64_t step)
@@ -287,8 +295,9 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         if (m.p.bucket != msgs[0].p.bucket) return DQ_ERR_UNSUPPORTED;
         if (!half_dithered && (m.p.dither_bits == 16u) != (msgs[0].p.dither_bits == 16u)) return DQ_ERR_UNSUPPORTED;
         dq::DecWorker& d = a.w[w];
-        d.packed = m.packed;
-        d.scale = m.scale;
+        // addresses of the (virtual) whole-gradient buffers: see DecodeArgs
+        d.packed = virtual_base(m.packed, first_element / 32u * m.p.bits);
+        d.scale = virtual_base(m.scale, first_element / m.p.bucket);
         fill_philox(d.ps, m.seed, m.worker, step);
         d.bits = m.p.bits;
         if (m.kind == DQ_KIND_DQSG) {
@@ -324,18 +333,18 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
         if (!aligned16(msgs[w].packed) || !aligned16(msgs[w].scale)) return DQ_ERR_ALIGNMENT;
     }
-    a.side = (any_nested && !running) ? side_info : nullptr;
-    a.out = out_avg;
+    a.side = (any_nested && !running) ? virtual_base(side_info, first_element) : nullptr;
+    a.out = virtual_base(out_avg, first_element);
     a.status = status_word;
-    a.n = n;
-    a.rows = (n + 31u) / 32u;
-    a.row_offset = first_element / 32u;
+    a.n = first_element + n;
+    a.rows = (first_element + n + 31u) / 32u;
+    a.first_row = first_element / 32u;
     a.W = W;
     a.rows_per_bucket = msgs[0].p.bucket / 32u;
     a.half_bias_bits = 0x4A800000u;
     a.Wf = (float)W;
     a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
-    const uint64_t grid64 = (a.rows + dq::kDecThreads - 1u) / dq::kDecThreads;
+    const uint64_t grid64 = (a.rows - a.first_row + dq::kDecThreads - 1u) / dq::kDecThreads;
     if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
     const bool d16 = (msgs[0].p.dither_bits == 16u);
     const uint32_t grid = (uint32_t)grid64;

@@ -39,10 +39,13 @@ struct DecodeArgs {
     const float* side;
     float* out;
     uint32_t* status;
-    uint64_t n;
-    uint64_t rows;            // ceil(n / 32)
-    uint64_t row_offset;      // index of out[0]'s row in the whole gradient (0 unless a bucket range is decoded):
-                              // only the dither counters see it
+    // A call may cover the elements [first, n) of a longer gradient (first a multiple of the bucket size, 0 for a
+    // whole gradient).  Rows, elements and buckets are then numbered as in the whole gradient -- which is what the
+    // dither counters need -- and every pointer below is the buffer's address minus the range's offset, so that
+    // "pointer + global index" lands in the caller's buffer.
+    uint64_t n;               // end of the range (element index)
+    uint64_t rows;            // ceil(n / 32): end of the range (row index)
+    uint64_t first_row;       // first / 32
     uint32_t W;
     uint32_t rows_per_bucket; // B / 32
     uint32_t half_bias_bits;  // 0x4A800000 (bit pattern of 2^22), passed in so that it lives in a register
@@ -196,11 +199,11 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t
             if (DITH == 0) {
                 f = 1.5f;
             } else if (DITH == 16) {
-                ctr[0] = (uint32_t)((i + 32u * args.row_offset) >> 3);
+                ctr[0] = (uint32_t)(i >> 3);
                 philox4x32_10_xN<1>(ctr, wk.ps, rnd);
                 f = dither16_f12(rnd[0][(i & 7u) >> 1], (int)(i & 1u));
             } else {
-                ctr[0] = (uint32_t)((i + 32u * args.row_offset) >> 2);
+                ctr[0] = (uint32_t)(i >> 2);
                 philox4x32_10_xN<1>(ctr, wk.ps, rnd);
                 f = dither_f12(rnd[0][i & 3u]);
             }
@@ -241,7 +244,7 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     __shared__ __align__(16) float side_tile[RUN ? 4 : kDecThreads * 32];
     grid_dependency_wait();
     grid_dependency_launch_next();
-    const uint64_t row0 = (uint64_t)blockIdx.x * blockDim.x;
+    const uint64_t row0 = args.first_row + (uint64_t)blockIdx.x * blockDim.x;
     if (!RUN && args.side != nullptr) {
         // kDecThreads rows x 8 pieces = 8 pieces per thread
 #pragma unroll
@@ -277,10 +280,10 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
         float kappa;
         load_worker_row(wk, row, bucket, cur, kappa);
         switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row + args.row_offset, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row + args.row_offset, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row + args.row_offset, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
-            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row + args.row_offset, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
         }
     }
 
