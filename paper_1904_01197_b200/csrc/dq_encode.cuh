@@ -333,9 +333,10 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         // B = 4096, 8192: the same, with two or four warps taking 2048 elements each and meeting once per bucket
         // to exchange their maxima.
         const uint32_t sub = warp % wpb;                 // this warp's 2048-element part of the bucket
-        for (uint64_t pair = first_tile; pair < args.num_units; pair += stride, ++k) {
+        // (unit indices stay far below 2^32 - stride: a unit is at least 2048 elements and n < 2^34)
+        for (uint32_t pair = first_tile; pair < args.num_units; pair += stride, ++k) {
             const uint32_t par = k & 1u;
-            const uint64_t part = pair * wpb + sub;      // index of this warp's 2048 elements in the gradient
+            const uint32_t part = pair * wpb + sub;      // index of this warp's 2048 elements in the gradient
             float x[32];
             float mx = 0.0f;
 #pragma unroll 1
@@ -389,7 +390,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    const uint64_t next = pair + stride;
+                    const uint32_t next = pair + stride;
                     if (next < args.num_units) {
                         mbar_expect_tx(my_bar + 8u * half, (uint32_t)kWarpTileBytes);
                         tma_load_rows(my_smem + half * kWarpTileBytes, &tmap, my_bar + 8u * half,
@@ -397,7 +398,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                     }
                 }
                 const float a = bucket_gain(args.gain_num, mx);
-                const uint32_t row = (uint32_t)part * 64u + half * 32u + lane;
+                const uint32_t row = part * 64u + half * 32u + lane;
                 uint32_t out[BITS];
                 encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
                 store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
