@@ -189,6 +189,24 @@ def ndqsg_encode(grad: torch.Tensor, seed: int, worker: int, step: int, params: 
     return _encode(lib().ndqsg_encode, "ndqsg_encode", grad, seed, worker, step, params, out_packed, out_scale, stream)
 
 
+def bucket_ranges(n: int, bucket: int, parts: int):
+    """Cuts [0, n) into `parts` consecutive bucket-aligned ranges of nearly equal bucket counts (host arithmetic).
+
+    Returns [(first_element, count), ...]; ranges at the end may be empty when there are fewer buckets than parts.
+    Feed them to the *_range calls: one range per GPU, per transfer chunk or per layer group.
+    """
+    if n < 0 or bucket <= 0 or parts <= 0:
+        raise ValueError("bucket_ranges: n >= 0, bucket > 0 and parts > 0 are required")
+    nb = -(-n // bucket)
+    out = []
+    for r in range(parts):
+        b0 = nb * r // parts
+        b1 = nb * (r + 1) // parts
+        lo, hi = min(n, b0 * bucket), min(n, b1 * bucket)
+        out.append((lo, hi - lo))
+    return out
+
+
 def _encode_range(fn, what, grad, first_element, seed, worker, step, params, out_packed, out_scale, stream):
     n = grad.numel()
     if out_packed is None or out_scale is None:
