@@ -115,3 +115,41 @@ def test_a_range_must_start_at_a_bucket_boundary(dq):
     with pytest.raises(dq.DqError) as e:                       # beyond the supported length
         dq.dqsg_encode_range(g, (1 << 34), 1, 0, 0, p)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("bucket,bits_mix", [(2048, (3, 2, 2)), (96, (1, 5, 3))])
+def test_host_buffer_decode_of_a_long_gradient(dq, oracle, bucket, bits_mix):
+    # the host-buffer decode of a few million elements: same bits as the device entry point on the whole vector,
+    # and as the oracle on sampled bucket ranges (encoded and decoded with their global offset)
+    rng = np.random.default_rng(bucket)
+    n = (1 << 21) + 37 * bucket + 19
+    step = 12
+    side = rng.standard_normal(n).astype(np.float32)
+    specs = [WorkerSpec(DQSG, bits_mix[0], 0, seed=801), WorkerSpec(NDQSG, bits_mix[1], 0, 1 << bits_mix[1], 4.0, 1.0, 802),
+             WorkerSpec(NDQSG, bits_mix[2], 0, (1 << bits_mix[2]) - 1 if bits_mix[2] > 1 else 2, 3.0, 0.9, 803)]
+    dev_msgs, host_msgs, keep = [], [], []
+    grads = []
+    for w, sp in enumerate(specs):
+        g = (side + 0.1 * rng.standard_normal(n)).astype(np.float32)
+        grads.append(g)
+        pk, sc = gpu_encode(dq, torch, torch.from_numpy(g).cuda(), sp, w, step, bucket)
+        dev_msgs.append(gpu_msg(dq, pk, sc, sp, w, bucket))
+        hpk, hsc = pk.cpu().pin_memory(), sc.cpu().pin_memory()
+        host_msgs.append(dq.Message(hpk, hsc, sp.seed, w, sp.kind, spec_params(dq, sp, bucket)))
+        keep += [pk, sc, hpk, hsc]
+    whole = dq.ndqsg_decode_aggregate(dev_msgs, n, step, torch.from_numpy(side).cuda())[:n].cpu().numpy()
+    out = torch.empty(n, dtype=torch.float32).pin_memory()
+    ws = torch.empty(dq.decode_workspace_bytes(host_msgs, n, True), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                   # twice: the staging area is reused
+        out.zero_()
+        dq.ndqsg_decode_aggregate_host(host_msgs, n, step, torch.from_numpy(side).pin_memory(), out, ws)
+        assert np.array_equal(out.numpy().view(np.uint32), whole.view(np.uint32))
+    for b0 in (0, (n // bucket) // 2, n // bucket - 1):  # oracle on three bucket pairs, the ragged end included
+        lo, hi = b0 * bucket, min(n, (b0 + 2) * bucket)
+        om = []
+        for w, sp in enumerate(specs):
+            opk, osc = oracle_encode(oracle, grads[w][lo:hi], sp, w, step, bucket, i0=lo)
+            om.append(oracle_msg(oracle, opk, osc, sp, w, bucket))
+        ref = oracle.decode_aggregate(om, hi - lo, step, side_info=side[lo:hi], i0=lo)
+        assert_fp32_close(out.numpy()[lo:hi], ref, f"buckets from {b0}")
+    assert dq.device_error_flags() == 0
