@@ -252,7 +252,17 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     const uint32_t slots = (uint32_t)dq::kEncCtasPerSm * (uint32_t)sms;   // resident CTAs
     uint32_t plain = 0;
     if (rest > 0) {
-        const uint64_t want = (rest + dq::kConsumerWarps - 1u) / dq::kConsumerWarps;
+        // buckets of at most 32 rows: a warp takes a window of whole buckets; up to 128 rows: a warp per bucket;
+        // larger ones: a CTA per bucket
+        uint64_t want = rest;
+        if (B <= 1024u) {
+            const uint64_t rpb = B / 32u, rows_per_window = (32u / rpb) * rpb;
+            const uint64_t rest_rows = (n + 31u) / 32u - a.first_bucket * rpb;
+            a.plain_windows = (rest_rows + rows_per_window - 1u) / rows_per_window;
+            want = (a.plain_windows + dq::kConsumerWarps - 1u) / dq::kConsumerWarps;
+        } else if (B <= dq::kPlainWarpBucketMax) {
+            want = (rest + dq::kConsumerWarps - 1u) / dq::kConsumerWarps;           // a warp per bucket
+        }
         const uint64_t cap = (tiles > 0) ? (slots / 4u) : (4ull * slots);
         plain = (uint32_t)(want < cap ? want : cap);
         if (plain == 0u) plain = 1u;

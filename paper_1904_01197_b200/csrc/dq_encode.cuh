@@ -18,7 +18,9 @@
 // The units are dealt out round-robin over the warp groups of all CTAs.  The gradient is read from HBM exactly once.
 //
 // Everything else -- other bucket sizes, the part of the vector past the last whole tile, the ragged end --
-// is handled by plain-load code, one warp per bucket, in extra CTAs of the same launch.
+// is handled by plain-load code in extra CTAs of the same launch: buckets of at most 32 rows in warp windows of
+// whole buckets (one row per lane, segmented maximum over the lanes), buckets of up to 4096 elements one per warp,
+// larger ones one per CTA (a sweep for the maximum, then a second, cached sweep that quantizes).
 #pragma once
 
 #include "dq_device.cuh"
@@ -43,6 +45,8 @@ constexpr int kEncCtasPerSm = DQ_ENC_CTAS_PER_SM;
 constexpr size_t kEncSmemBytes = (size_t)kEncStages * kTileBytes + 1024;
 // Time HBM needs to deliver one warp's pipeline stages (8 KB) to each of the 148 SMs: 148 x 8 KB / 6.5 TB/s.
 constexpr uint32_t kFirstRequestSpacingNs = 190u;
+// Plain-load part: buckets up to 1024 elements are taken in warp windows, up to this size by one warp, above by a CTA.
+constexpr uint32_t kPlainWarpBucketMax = 4096u;
 
 struct EncodeArgs {
     const float* grad;
@@ -54,6 +58,7 @@ struct EncodeArgs {
     uint64_t num_words;      // total packed words of the gradient
     uint32_t num_units;      // work units of the tile path: max(B, 1024) elements each (see encode_kernel)
     uint32_t plain_ctas;     // the first plain_ctas CTAs run the plain-load part, the rest walk over the tiles
+    uint64_t plain_windows;  // B <= 1024: windows of whole buckets (at most 32 rows) in the plain-load part
     uint32_t bucket;         // B
     uint32_t bucket_log2;    // log2(B) on the tile path
     uint32_t lanes_per_bucket;  // B / 32 when B < 1024, else 32
@@ -197,54 +202,142 @@ __device__ __forceinline__ float bucket_gain(float num, float kappa)
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Plain-load part: one warp per bucket, any bucket size, ragged end.
+// Plain-load part: any bucket size, the part of the vector past the last whole tile, the ragged end.
 // ---------------------------------------------------------------------------------------------------
+
+// The `nvalid` (1..32) elements of row `grow` of the gradient, zero-filled.
+__device__ __forceinline__ void load_row_plain(const EncodeArgs& args, uint64_t grow, uint32_t nvalid, float (&x)[32])
+{
+    const float* g = args.grad + grow * 32u;
+    if (nvalid == 32u) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float4 v = reinterpret_cast<const float4*>(g)[c];
+            x[4 * c] = v.x; x[4 * c + 1] = v.y; x[4 * c + 2] = v.z; x[4 * c + 3] = v.w;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) x[e] = ((uint32_t)e < nvalid) ? g[e] : 0.0f;
+    }
+}
+
+// Quantizes and stores row `grow` (already in registers) with the bucket's gain `a`.
 template <int BITS, int MODE, int DITH>
-__device__ __forceinline__ void encode_bucket_plain(const EncodeArgs& args, uint64_t bucket, uint32_t lane)
+__device__ __forceinline__ void encode_store_row_plain(const EncodeArgs& args, const float (&x)[32], uint64_t grow,
+                                                       uint32_t nvalid, float a)
+{
+    uint32_t out[BITS];
+    encode_row<BITS, MODE, DITH>(x, (uint32_t)grow + args.row_offset, a, args, out);
+    uint32_t* dst = args.packed + grow * BITS;
+    if (nvalid == 32u) {
+        store_row_words<BITS>(dst, out);
+    } else {
+        // last row of the gradient: clear the codes of elements past the end, write only existing words
+        const uint32_t valid_bits = nvalid * BITS;
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) {
+            const int32_t keep = (int32_t)valid_bits - 32 * j;
+            if (keep <= 0) continue;
+            const uint32_t m = (keep >= 32) ? 0xFFFFFFFFu : ((1u << keep) - 1u);
+            if (grow * BITS + j < args.num_words) dst[j] = out[j] & m;
+        }
+    }
+}
+
+// Buckets of at most 32 rows: a warp takes a window of as many whole buckets as fit into 32 rows, one row per
+// lane; the maximum of a bucket is a segmented reduction over the lanes that hold its rows.
+template <int BITS, int MODE, int DITH>
+__device__ __forceinline__ void encode_window_plain(const EncodeArgs& args, uint64_t window, uint32_t lane)
+{
+    const uint32_t rpb = args.bucket >> 5;                     // rows per bucket (<= 32)
+    const uint32_t rows_per_window = (32u / rpb) * rpb;
+    const uint64_t total_rows = (args.n + 31u) >> 5;
+    const uint64_t grow = (args.first_bucket * rpb) + window * rows_per_window + lane;
+    const bool active = lane < rows_per_window && grow < total_rows;
+    const uint32_t nvalid = !active ? 0u : (args.n - grow * 32u < 32u) ? (uint32_t)(args.n - grow * 32u) : 32u;
+    float x[32];
+    float mx = 0.0f;
+    if (active) {
+        load_row_plain(args, grow, nvalid, x);
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) mx = max3_abs(mx, x[e], x[e + 1]);
+    }
+    // lanes of one bucket are adjacent: take the neighbour's maximum while it belongs to the same bucket
+    const uint32_t seg = lane / rpb;
+#pragma unroll
+    for (uint32_t off = 1; off < 32u; off <<= 1) {
+        const float up = __shfl_up_sync(0xFFFFFFFFu, mx, off);
+        const float down = __shfl_down_sync(0xFFFFFFFFu, mx, off);
+        if (lane >= off && (lane - off) / rpb == seg) mx = fmaxf(mx, up);
+        if (lane + off < 32u && (lane + off) / rpb == seg) mx = fmaxf(mx, down);
+    }
+    if (!active) return;
+    if (lane % rpb == 0u) args.scale[grow / rpb] = mx;
+    encode_store_row_plain<BITS, MODE, DITH>(args, x, grow, nvalid, bucket_gain(args.gain_num, mx));
+}
+
+// Buckets of 33 to 128 rows: one warp per bucket (a first sweep for the maximum, then one row per lane at a time).
+template <int BITS, int MODE, int DITH>
+__device__ __forceinline__ void encode_bucket_warp_plain(const EncodeArgs& args, uint64_t bucket, uint32_t lane)
 {
     const uint64_t lo = bucket * args.bucket;
     const uint32_t len = (uint32_t)((args.n - lo < args.bucket) ? (args.n - lo) : args.bucket);
     const float* g = args.grad + lo;
-
     float mx = 0.0f;
-    for (uint32_t i = lane; i < len; i += 32u) mx = fmaxf(mx, fabsf(g[i]));
+    const uint32_t quads = len >> 2;
+    for (uint32_t q = lane; q < quads; q += 32u) {
+        const float4 v = reinterpret_cast<const float4*>(g)[q];
+        mx = max3_abs(max3_abs(mx, v.x, v.y), v.z, v.w);
+    }
+    for (uint32_t i = (quads << 2) + lane; i < len; i += 32u) mx = fmaxf(mx, fabsf(g[i]));
 #pragma unroll
     for (uint32_t off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
     if (lane == 0) args.scale[bucket] = mx;
     const float a = bucket_gain(args.gain_num, mx);
-
     const uint32_t rows = (len + 31u) >> 5;
     for (uint32_t r = lane; r < rows; r += 32u) {
-        const uint32_t base = r * 32u;
-        const uint32_t nvalid = (len - base < 32u) ? (len - base) : 32u;
-        float x[32];
-        if (nvalid == 32u) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float4 v = reinterpret_cast<const float4*>(g + base)[c];
-                x[4 * c] = v.x; x[4 * c + 1] = v.y; x[4 * c + 2] = v.z; x[4 * c + 3] = v.w;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) x[e] = ((uint32_t)e < nvalid) ? g[base + e] : 0.0f;
-        }
-        uint32_t out[BITS];
+        const uint32_t nvalid = (len - r * 32u < 32u) ? (len - r * 32u) : 32u;
         const uint64_t grow = (lo >> 5) + r;
-        encode_row<BITS, MODE, DITH>(x, (uint32_t)grow + args.row_offset, a, args, out);
-        uint32_t* dst = args.packed + grow * BITS;
-        if (nvalid == 32u) {
-            store_row_words<BITS>(dst, out);
-        } else {
-            // last row of the gradient: clear the codes of elements past the end, write only existing words
-            const uint32_t valid_bits = nvalid * BITS;
+        float x[32];
+        load_row_plain(args, grow, nvalid, x);
+        encode_store_row_plain<BITS, MODE, DITH>(args, x, grow, nvalid, a);
+    }
+}
+
+// Buckets of more than 128 rows: the whole CTA takes one bucket; a first sweep finds the maximum, a second one
+// (served by the caches) quantizes one row per lane at a time.
+template <int BITS, int MODE, int DITH>
+__device__ __forceinline__ void encode_bucket_cta_plain(const EncodeArgs& args, uint64_t bucket, float* cta_max)
+{
+    const uint64_t lo = bucket * args.bucket;
+    const uint32_t len = (uint32_t)((args.n - lo < args.bucket) ? (args.n - lo) : args.bucket);
+    const float* g = args.grad + lo;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+
+    float mx = 0.0f;
+    const uint32_t quads = len >> 2;
+    for (uint32_t q = threadIdx.x; q < quads; q += (uint32_t)kEncThreads) {
+        const float4 v = reinterpret_cast<const float4*>(g)[q];
+        mx = max3_abs(max3_abs(mx, v.x, v.y), v.z, v.w);
+    }
+    for (uint32_t i = (quads << 2) + threadIdx.x; i < len; i += (uint32_t)kEncThreads) mx = fmaxf(mx, fabsf(g[i]));
 #pragma unroll
-            for (int j = 0; j < BITS; ++j) {
-                const int32_t keep = (int32_t)valid_bits - 32 * j;
-                if (keep <= 0) continue;
-                const uint32_t m = (keep >= 32) ? 0xFFFFFFFFu : ((1u << keep) - 1u);
-                if (grow * BITS + j < args.num_words) dst[j] = out[j] & m;
-            }
-        }
+    for (uint32_t off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+    __syncthreads();                                           // the previous bucket's maxima have been read
+    if (lane == 0) cta_max[warp] = mx;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; ++w) mx = fmaxf(mx, cta_max[w]);
+    if (threadIdx.x == 0) args.scale[bucket] = mx;
+    const float a = bucket_gain(args.gain_num, mx);
+
+    const uint32_t rows = (len + 31u) >> 5;
+    for (uint32_t r = threadIdx.x; r < rows; r += (uint32_t)kEncThreads) {
+        const uint32_t nvalid = (len - r * 32u < 32u) ? (len - r * 32u) : 32u;
+        const uint64_t grow = (lo >> 5) + r;
+        float x[32];
+        load_row_plain(args, grow, nvalid, x);
+        encode_store_row_plain<BITS, MODE, DITH>(args, x, grow, nvalid, a);
     }
 }
 
@@ -271,10 +364,21 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
 
     if (blockIdx.x < args.plain_ctas) {
         grid_dependency_wait();
-        // plain-load part: warps take buckets round-robin over these CTAs
-        for (uint64_t b = args.first_bucket + (uint64_t)blockIdx.x * kConsumerWarps + warp;
-             b < args.num_buckets; b += (uint64_t)args.plain_ctas * kConsumerWarps)
-            encode_bucket_plain<BITS, MODE, DITH>(args, b, lane);
+        if (args.bucket <= 1024u) {
+            // windows of whole buckets (at most 32 rows), one per warp, round-robin over these CTAs
+            for (uint64_t w = (uint64_t)blockIdx.x * kConsumerWarps + warp; w < args.plain_windows;
+                 w += (uint64_t)args.plain_ctas * kConsumerWarps)
+                encode_window_plain<BITS, MODE, DITH>(args, w, lane);
+        } else if (args.bucket <= kPlainWarpBucketMax) {
+            // one bucket per warp at a time
+            for (uint64_t b = args.first_bucket + (uint64_t)blockIdx.x * kConsumerWarps + warp;
+                 b < args.num_buckets; b += (uint64_t)args.plain_ctas * kConsumerWarps)
+                encode_bucket_warp_plain<BITS, MODE, DITH>(args, b, lane);
+        } else {
+            // one bucket per CTA at a time
+            for (uint64_t b = args.first_bucket + blockIdx.x; b < args.num_buckets; b += args.plain_ctas)
+                encode_bucket_cta_plain<BITS, MODE, DITH>(args, b, &warp_max[0][0]);
+        }
         return;
     }
 
