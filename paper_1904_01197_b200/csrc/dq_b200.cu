@@ -349,6 +349,10 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.n = first_element + n;
     a.rows = (first_element + n + 31u) / 32u;
     a.first_row = first_element / 32u;
+    {
+        const int sms_now = device_sm_count();
+        a.prefetch_blocks = (sms_now > 0) ? (uint32_t)(dq::kDecMinBlocks * sms_now) : 0u;
+    }
     a.W = W;
     a.rows_per_bucket = msgs[0].p.bucket / 32u;
     a.half_bias_bits = 0x4A800000u;

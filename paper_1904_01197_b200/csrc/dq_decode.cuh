@@ -46,6 +46,7 @@ struct DecodeArgs {
     uint64_t n;               // end of the range (element index)
     uint64_t rows;            // ceil(n / 32): end of the range (row index)
     uint64_t first_row;       // first / 32
+    uint32_t prefetch_blocks; // distance, in 128-row blocks, of the L2 prefetch (0 = none)
     uint32_t W;
     uint32_t rows_per_bucket; // B / 32
     uint32_t half_bias_bits;  // 0x4A800000 (bit pattern of 2^22), passed in so that it lives in a register
@@ -245,6 +246,21 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     grid_dependency_wait();
     grid_dependency_launch_next();
     const uint64_t row0 = args.first_row + (uint64_t)blockIdx.x * blockDim.x;
+    {
+        // Ask the L2 for what the CTA that runs `prefetch_blocks` blocks later (about one wave of resident CTAs)
+        // will load first: its side information and every message's words, so that those loads find their lines
+        // in the L2 instead of waiting for HBM.
+        const uint64_t frow0 = row0 + (uint64_t)args.prefetch_blocks * kDecThreads;
+        if (frow0 + threadIdx.x < args.rows) {
+            if (!RUN && args.side != nullptr) prefetch_l2(args.side + (frow0 + threadIdx.x) * 32u);
+        }
+        const uint32_t lane = threadIdx.x & 31u;
+        for (uint32_t w = threadIdx.x >> 5; w < args.W; w += (uint32_t)kDecThreads / 32u) {
+            const uint64_t first_word = frow0 * args.w[w].bits + 32u * lane;          // lines of 32 words
+            if (lane < 4u * args.w[w].bits && first_word < args.rows * args.w[w].bits)
+                prefetch_l2(args.w[w].packed + first_word);
+        }
+    }
     if (!RUN && args.side != nullptr) {
         // kDecThreads rows x 8 pieces = 8 pieces per thread
 #pragma unroll
