@@ -44,14 +44,14 @@ DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 
 # multiplies / multiply-adds, everything else).  Their scheduler cost is taken from the issue probe
 # (profiles/issue_cost_probe_b200.md): 4.4 cycles per wide multiply with one other instruction hidden behind it,
 # 1 cycle per fp32 instruction, 2 cycles for the rest; the classes add up.
-DEC_MIX = {32: (4.32, 9.82, 12.23), 16: (2.18, 9.82, 9.59)}
+DEC_MIX = {32: (4.34, 9.82, 12.52), 16: (2.20, 9.82, 9.88)}
 ISSUE_CYCLES_WIDE, ISSUE_CYCLES_FP32, ISSUE_CYCLES_OTHER = 4.4, 1.0, 2.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
 # profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
 NCU_TRAFFIC = {
     ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_543_616,    # profiles/encode_kernel_ndqsg_resnet50.md
     ("encode", "ndqsg_resnet50", 25_557_032, 3): 106_651_648,
-    ("decode", "ndqsg_resnet50", 25_557_032): 219_680_512,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
+    ("decode", "ndqsg_resnet50", 25_557_032): 223_945_472,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
 }
 
 
