@@ -351,7 +351,8 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     a.first_row = first_element / 32u;
     {
         const int sms_now = device_sm_count();
-        a.prefetch_blocks = (sms_now > 0) ? (uint32_t)(dq::kDecMinBlocks * sms_now) : 0u;
+        // one block per SM ahead: 16 to 200 blocks measured alike, a whole wave (4 per SM) or more is too far
+        a.prefetch_blocks = (sms_now > 0) ? (uint32_t)sms_now : 0u;
     }
     a.W = W;
     a.rows_per_bucket = msgs[0].p.bucket / 32u;

@@ -247,8 +247,8 @@ decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
     grid_dependency_launch_next();
     const uint64_t row0 = args.first_row + (uint64_t)blockIdx.x * blockDim.x;
     {
-        // Ask the L2 for what the CTA that runs `prefetch_blocks` blocks later (about one wave of resident CTAs)
-        // will load first: its side information and every message's words, so that those loads find their lines
+        // Ask the L2 for what the CTA that runs `prefetch_blocks` blocks later (one block per SM ahead) will load
+        // first: its side information and every message's words, so that those loads find their lines
         // in the L2 instead of waiting for HBM.
         const uint64_t frow0 = row0 + (uint64_t)args.prefetch_blocks * kDecThreads;
         if (frow0 + threadIdx.x < args.rows) {
