@@ -67,8 +67,19 @@ typedef struct {
     float    fine_M;    /* NDQSG: M1 = 1/Delta_1 in units of kappa, 0 < alpha*M1 <= 2^20.                 */
     float    alpha;     /* NDQSG: shrinkage, 0 < alpha <= 1; 0 selects 1.                                 */
     uint32_t dither_bits; /* random bits per dither value: 32 (0 selects it) or 16, see above              */
-    uint32_t reserved;  /* set to 0                                                                       */
+    uint32_t flags;     /* DQ_FLAG_* bits, 0 for none                                                     */
 } dq_params;
+
+/*
+ * DQ_FLAG_INPUT_READY (encoders only; ignored elsewhere).  By default an encode kernel touches no memory
+ * before the previous kernel of its stream has completed.  With this flag the caller declares that `grad`
+ * was completely written before that previous kernel was launched and is not written by it -- the usual case
+ * when a gradient produced by the backward pass is encoded after some unrelated kernel, or when several
+ * gradients are encoded back to back.  The encoder then requests and quantizes its first tiles while the
+ * previous kernel is still draining; its stores to out_packed and out_scale still wait for that kernel to
+ * complete, so outputs may be shared with it.  Results are identical with and without the flag.
+ */
+#define DQ_FLAG_INPUT_READY 0x1u
 
 /* One worker's message as the decoder sees it. */
 typedef struct {

@@ -18,6 +18,7 @@ DQ_KIND_NDQSG = 1
 DQ_WARN_NONFINITE_SCALE = 0x1
 DQ_ERR_COPY_TIMEOUT = 0x2
 DQ_WARN_CODE_RANGE = 0x4
+DQ_FLAG_INPUT_READY = 0x1
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libdq_b200.so"
 
@@ -31,7 +32,7 @@ class DqError(RuntimeError):
 class DqParams(C.Structure):
     _fields_ = [("bucket", C.c_uint32), ("bits", C.c_uint32), ("levels", C.c_uint32),
                 ("coarse_K", C.c_uint32), ("fine_M", C.c_float), ("alpha", C.c_float),
-                ("dither_bits", C.c_uint32), ("reserved", C.c_uint32)]
+                ("dither_bits", C.c_uint32), ("flags", C.c_uint32)]
 
 
 class DqMsg(C.Structure):
@@ -136,8 +137,8 @@ def _host_ptr(t, dtype, what: str) -> Optional[int]:
 
 
 def make_params(bucket: int, bits: int, levels: int = 0, coarse_K: int = 0, fine_M: float = 0.0,
-                alpha: float = 0.0, dither_bits: int = 0) -> DqParams:
-    return DqParams(bucket, bits, levels, coarse_K, fine_M, alpha, dither_bits, 0)
+                alpha: float = 0.0, dither_bits: int = 0, flags: int = 0) -> DqParams:
+    return DqParams(bucket, bits, levels, coarse_K, fine_M, alpha, dither_bits, flags)
 
 
 class Message:

@@ -1,19 +1,23 @@
-"""Builds the CUDA library in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
+"""Builds the CUDA library in-tree with nvcc for sm_100a (cross-compiles without a GPU).
+
+The kernels are templates with many instantiations; they are spread over translation units (one per encoder
+mode and dither width, one per decoder variant) that are compiled in parallel and linked into one shared library.
+"""
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 from pathlib import Path
 
 PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "lib" / "libdq_b200.so"
-SOURCES = [CSRC / "dq_b200.cu"]
-PROBE_SOURCE = CSRC / "issue_probe.cu"          # stand-alone program, see issue_probe.py
-PROBE = PKG / "lib" / "dq_issue_probe"
-DEPS = sorted(f for f in CSRC.glob("*.cu*") if f != PROBE_SOURCE) + [ROOT / "include" / "dq.h"]
+OBJ = PKG / "lib" / "obj"
+DEPS = sorted(CSRC.glob("*.cu*")) + sorted(CSRC.glob("*.h")) + [ROOT / "include" / "dq.h"]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3",
@@ -21,14 +25,29 @@ NVCC_FLAGS = [
     "-lineinfo",
     "--fmad=false",          # every fused multiply-add in the kernels is written explicitly
     "-Xcompiler", "-fPIC",
-    "-cudart", "static",
-    "-shared",
 ]
+
+# (object name, source, extra defines)
+UNITS = [("dq_b200", "dq_b200.cu", [])]
+UNITS += [(f"enc_m{m}_d{d}", "dq_encode_inst.cu", [f"-DDQ_INST_MODE={m}", f"-DDQ_INST_DITH={d}"])
+          for m in (0, 1, 2, 3) for d in (32, 16)]
+UNITS += [(f"dec_d{d}_r{r}", "dq_decode_inst.cu", [f"-DDQ_INST_DITH={d}", f"-DDQ_INST_RUN={r}"])
+          for d, r in ((32, 0), (32, 1), (16, 0), (16, 1), (0, 0))]
 
 
 def nvcc_path() -> str:
     cand = os.environ.get("NVCC") or "/usr/local/cuda/bin/nvcc"
     return cand if Path(cand).exists() else "nvcc"
+
+
+def source_hash() -> str:
+    """Content hash of everything the library is built from (sources, headers, flags)."""
+    h = hashlib.sha256()
+    for f in DEPS:
+        h.update(f.name.encode())
+        h.update(f.read_bytes())
+    h.update(" ".join(NVCC_FLAGS).encode())
+    return h.hexdigest()[:16]
 
 
 def stale() -> bool:
@@ -38,32 +57,30 @@ def stale() -> bool:
     return any(d.stat().st_mtime > t for d in DEPS)
 
 
+def _compile(unit, verbose: bool) -> Path:
+    name, src, defs = unit
+    obj = OBJ / f"{name}.o"
+    cmd = [nvcc_path(), *NVCC_FLAGS, *defs, f"-I{ROOT / 'include'}", f"-I{CSRC}", "-c", "-o", str(obj),
+           str(CSRC / src)]
+    if verbose:
+        cmd += ["-Xptxas", "-v"]
+    subprocess.run(cmd, check=True)
+    return obj
+
+
 def build(force: bool = False, verbose: bool = False) -> Path:
     if not force and not stale():
         return LIB
-    LIB.parent.mkdir(parents=True, exist_ok=True)
+    OBJ.mkdir(parents=True, exist_ok=True)
+    jobs = int(os.environ.get("DQ_BUILD_JOBS", "0")) or min(len(UNITS), os.cpu_count() or 1)
+    with ThreadPoolExecutor(max_workers=jobs) as pool:
+        objs = list(pool.map(lambda u: _compile(u, verbose), UNITS))
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [nvcc_path(), *NVCC_FLAGS, f"-I{ROOT / 'include'}", f"-I{CSRC}", "-o", str(tmp)]
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [str(s) for s in SOURCES]
-    subprocess.run(cmd, check=True)
+    subprocess.run([nvcc_path(), "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
+                    "-o", str(tmp), *[str(o) for o in objs]], check=True)
     os.replace(tmp, LIB)
     return LIB
 
 
-def build_probe(force: bool = False) -> Path:
-    """Compiles the issue-cost probe (a stand-alone executable that uses no library code)."""
-    if not force and PROBE.exists() and PROBE.stat().st_mtime >= PROBE_SOURCE.stat().st_mtime:
-        return PROBE
-    PROBE.parent.mkdir(parents=True, exist_ok=True)
-    tmp = PROBE.with_suffix(f".{os.getpid()}.tmp")
-    subprocess.run([nvcc_path(), "-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-                    "-cudart", "static", "-o", str(tmp), str(PROBE_SOURCE)], check=True)
-    os.replace(tmp, PROBE)
-    return PROBE
-
-
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
-    print(build_probe(force="--force" in sys.argv))

@@ -9,10 +9,17 @@
 
 #include "dq_decode.cuh"
 #include "dq_encode.cuh"
+#include "dq_launch.h"
 #include "dq_stats.cuh"
 #include "dq_ternary.cuh"
 
+// The device's error word: kernels OR DQ_ERR_* bits into it through the address they are given.  In host code
+// the name is a handle for the runtime, not an address.
+static __device__ unsigned int g_dq_error_flags = 0u;
+
 namespace {
+
+using dq::launch_overlapped;
 
 std::atomic<uint64_t> g_launches{0};
 
@@ -122,63 +129,37 @@ bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t b
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Launch with programmatic stream serialization allowed: the kernels of this library all begin with
-// griddepcontrol.wait (nothing is read or written before the previous kernel of the stream has completed and
-// flushed), so letting the next launch start while this one drains only hides launch latency.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_overlapped(void (*kernel)(KArgs...), uint32_t grid, uint32_t block, size_t smem, cudaStream_t st,
-                              Args&&... args)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
-}
+constexpr int kMaxDevices = 64;
 
-template <int MODE, int BITS, int DITH>
-cudaError_t launch_encode_one(const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid, cudaStream_t st)
+// Device address of g_dq_error_flags on the current device; looked up once per device.
+unsigned int* error_flags_address()
 {
-    auto k = dq::encode_kernel<BITS, MODE, DITH>;
-    static bool configured[64] = {};        // the attribute is per device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dq::kEncSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured[dev] = true;
+    static std::mutex mu;
+    static unsigned int* addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_dq_error_flags) != cudaSuccess) return nullptr;
+        addr[dev] = static_cast<unsigned int*>(ptr);
     }
-    return launch_overlapped(k, grid, (uint32_t)dq::kEncThreads, dq::kEncSmemBytes, st, map, a);
+    return addr[dev];
 }
 
-template <int MODE, int DITH>
-cudaError_t launch_encode_bits(uint32_t bits, const CUtensorMap& map, const dq::EncodeArgs& a, uint32_t grid,
-                               cudaStream_t st)
-{
-    switch (bits) {
-        case 1: return launch_encode_one<MODE, 1, DITH>(map, a, grid, st);
-        case 2: return launch_encode_one<MODE, 2, DITH>(map, a, grid, st);
-        case 3: return launch_encode_one<MODE, 3, DITH>(map, a, grid, st);
-        case 4: return launch_encode_one<MODE, 4, DITH>(map, a, grid, st);
-        case 5: return launch_encode_one<MODE, 5, DITH>(map, a, grid, st);
-        case 6: return launch_encode_one<MODE, 6, DITH>(map, a, grid, st);
-        case 7: return launch_encode_one<MODE, 7, DITH>(map, a, grid, st);
-        default: return launch_encode_one<MODE, 8, DITH>(map, a, grid, st);
-    }
-}
-
-template <int MODE>
-cudaError_t launch_encode(uint32_t bits, bool dither16, const CUtensorMap& map, const dq::EncodeArgs& a,
+cudaError_t launch_encode(int mode, uint32_t bits, bool dither16, const CUtensorMap& map, const dq::EncodeArgs& a,
                           uint32_t grid, cudaStream_t st)
 {
-    return dither16 ? launch_encode_bits<MODE, 16>(bits, map, a, grid, st)
-                    : launch_encode_bits<MODE, 32>(bits, map, a, grid, st);
+    switch (mode * 2 + (dither16 ? 1 : 0)) {
+        case 0: return dq::launch_encode_m0_d32(bits, map, a, grid, st);
+        case 1: return dq::launch_encode_m0_d16(bits, map, a, grid, st);
+        case 2: return dq::launch_encode_m1_d32(bits, map, a, grid, st);
+        case 3: return dq::launch_encode_m1_d16(bits, map, a, grid, st);
+        case 4: return dq::launch_encode_m2_d32(bits, map, a, grid, st);
+        case 5: return dq::launch_encode_m2_d16(bits, map, a, grid, st);
+        case 6: return dq::launch_encode_m3_d32(bits, map, a, grid, st);
+        default: return dq::launch_encode_m3_d16(bits, map, a, grid, st);
+    }
 }
 
 dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t seed, uint32_t worker,
@@ -213,15 +194,19 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
         a.gain_num = a.shift;
         a.kmax = (float)(L - 1u);
     } else {
-        // The power-of-two path keeps the low `bits` bits of the index when bits divides 32 (K = 2^bits) and masks
-        // with K - 1 otherwise; a power of two below 2^bits with such a width takes the general path.
-        const bool low_bits_are_the_coset = (p->coarse_K == (1u << p->bits)) || (32u % p->bits) != 0u;
-        mode = (is_pow2(p->coarse_K) && low_bits_are_the_coset) ? dq::kEncNdqsgPow2 : dq::kEncNdqsgAnyK;
+        // K = 2^bits: the coset is the low `bits` bits of the fine index; a smaller power of two: one mask more;
+        // any other K: a modulo
+        mode = (p->coarse_K == (1u << p->bits)) ? dq::kEncNdqsgPow2
+               : is_pow2(p->coarse_K)           ? dq::kEncNdqsgPow2Mask
+                                                : dq::kEncNdqsgAnyK;
         a.gain_num = alpha * p->fine_M;
         a.K = p->coarse_K;
         a.K_offset = ((4194304u + p->coarse_K - 1u) / p->coarse_K) * p->coarse_K;
     }
     fill_philox(a.ps, seed, worker, step);
+    a.early_read = (p->flags & DQ_FLAG_INPUT_READY) ? 1u : 0u;
+    a.error_flags = error_flags_address();
+    if (!a.error_flags) return DQ_ERR_CUDA;
 
     // power-of-two buckets up to 8192: whole work units (a bucket, or 1024 elements for smaller buckets) go
     // through the tile path of the kernel, the rest (and every other bucket size) through its plain-load part,
@@ -277,12 +262,8 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     }
     // the spacing only pays when the first requests of all resident warps saturate HBM
     a.request_spacing_ns = (uint32_t)((uint64_t)dq::kFirstRequestSpacingNs * tile_ctas / slots);
-    cudaError_t e;
     const bool d16 = (p->dither_bits == 16u);
-    if (mode == dq::kEncDqsg) e = launch_encode<dq::kEncDqsg>(p->bits, d16, map, a, plain + tile_ctas, st);
-    else if (mode == dq::kEncNdqsgPow2) e = launch_encode<dq::kEncNdqsgPow2>(p->bits, d16, map, a, plain + tile_ctas, st);
-    else e = launch_encode<dq::kEncNdqsgAnyK>(p->bits, d16, map, a, plain + tile_ctas, st);
-    if (e != cudaSuccess) return DQ_ERR_CUDA;
+    if (launch_encode(mode, p->bits, d16, map, a, plain + tile_ctas, st) != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;
 }
@@ -364,15 +345,9 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     const bool d16 = (msgs[0].p.dither_bits == 16u);
     const uint32_t grid = (uint32_t)grid64;
     cudaError_t le;
-    if (half_dithered) {
-        le = launch_overlapped(dq::decode_aggregate_kernel<0, false>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
-    } else if (running && any_nested) {
-        if (d16) le = launch_overlapped(dq::decode_aggregate_kernel<16, true>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
-        else le = launch_overlapped(dq::decode_aggregate_kernel<32, true>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
-    } else {
-        if (d16) le = launch_overlapped(dq::decode_aggregate_kernel<16, false>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
-        else le = launch_overlapped(dq::decode_aggregate_kernel<32, false>, grid, (uint32_t)dq::kDecThreads, 0, st, a);
-    }
+    if (half_dithered) le = dq::launch_decode_d0_r0(a, grid, st);
+    else if (running && any_nested) le = d16 ? dq::launch_decode_d16_r1(a, grid, st) : dq::launch_decode_d32_r1(a, grid, st);
+    else le = d16 ? dq::launch_decode_d16_r0(a, grid, st) : dq::launch_decode_d32_r0(a, grid, st);
     if (le != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;
@@ -645,7 +620,6 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
 static __device__ __align__(256) unsigned char g_static_scratch[DQ_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_scratch_mutex;
 void* g_static_scratch_addr[kMaxDevices] = {};
 
@@ -688,8 +662,8 @@ dq_status dq_device_error_flags(uint32_t* out_flags)
     if (!out_flags) return DQ_ERR_INVALID_ARG;
     unsigned int v = 0u, zero = 0u;
     if (cudaDeviceSynchronize() != cudaSuccess) return DQ_ERR_CUDA;
-    if (cudaMemcpyFromSymbol(&v, dq::g_dq_error_flags, sizeof(v)) != cudaSuccess) return DQ_ERR_CUDA;
-    if (cudaMemcpyToSymbol(dq::g_dq_error_flags, &zero, sizeof(zero)) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, g_dq_error_flags, sizeof(v)) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpyToSymbol(g_dq_error_flags, &zero, sizeof(zero)) != cudaSuccess) return DQ_ERR_CUDA;
     *out_flags = v;
     return DQ_OK;
 }

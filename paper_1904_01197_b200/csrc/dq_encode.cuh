@@ -27,7 +27,9 @@
 
 namespace dq {
 
-enum EncMode : int { kEncDqsg = 0, kEncNdqsgPow2 = 1, kEncNdqsgAnyK = 2 };
+// kEncNdqsgPow2: K = 2^BITS, the coset is the low BITS bits of the fine index; kEncNdqsgPow2Mask: a smaller power
+// of two; kEncNdqsgAnyK: any K (a true modulo).
+enum EncMode : int { kEncDqsg = 0, kEncNdqsgPow2 = 1, kEncNdqsgAnyK = 2, kEncNdqsgPow2Mask = 3 };
 
 constexpr int kTileRows = 256;                     // rows a CTA holds per pipeline stage (8 warps x 32 rows, 32 KB)
 constexpr int kTileBytes = kTileRows * 128;
@@ -74,10 +76,12 @@ struct EncodeArgs {
                              // only the dither counters see it
     uint32_t sm_count;       // SMs of the device            } spacing of the first tile requests,
     uint32_t request_spacing_ns;   // see encode_kernel      } 0 when the grid does not fill the device
+    uint32_t early_read;     // the caller guarantees that grad was complete before the previous kernel of the stream
+                             // began: the tile path requests (and quantizes) its first tiles while that kernel
+                             // drains, and only its stores wait for it
+    unsigned int* error_flags;     // the library's per-device error word
     PhiloxStream ps;
 };
-
-__device__ unsigned int g_dq_error_flags = 0u;
 
 // max(m, |a|, |b|) in one instruction (three-input max, sm_100).
 __device__ __forceinline__ float max3_abs(float m, float a, float b)
@@ -87,24 +91,29 @@ __device__ __forceinline__ float max3_abs(float m, float a, float b)
     return d;
 }
 
-// ORs the low `nbits` bits of v into the row's bit stream at bit offset `bit` (all offsets are compile-time).
+// Appends the low BITS bits of `tb` to the row's bit stream.  `sr` is a 32-bit shift register whose top bits are
+// the most recent part of the stream: one funnel shift moves the older codes down and drops the bits of `tb` above
+// the code, so no masking and no shift of the code itself is needed.  `idx` (the element's position in the row) is
+// a compile-time constant after unrolling; a second funnel shift is only needed where a code straddles two words.
 template <int BITS>
-__device__ __forceinline__ void put_bits(uint32_t (&out)[BITS], int bit, int nbits, uint32_t v)
+__device__ __forceinline__ void push_code(uint32_t& sr, uint32_t tb, int idx, uint32_t (&out)[BITS])
 {
-    const int wi = bit >> 5;
-    const int sh = bit & 31;
-    out[wi] |= v << sh;
-    if (sh + nbits > 32) out[wi + 1] |= v >> (32 - sh);
+    const int end = (idx + 1) * BITS;                       // stream position after this code
+    const int over = end & 31;                              // bits of this code that belong to the next word
+    const bool completes = (end >> 5) != ((idx * BITS) >> 5);
+    if (completes && over != 0) out[(end >> 5) - 1] = __funnelshift_r(sr, tb, BITS - over);
+    sr = __funnelshift_r(sr, tb, BITS);
+    if (completes && over == 0) out[(end >> 5) - 1] = sr;
 }
 
-// DQSG: the rounded, clamped index of one element as an exact small float (0 .. L-1).
+// DQSG: bit pattern kMagicBits + k of one element, k the rounded, clamped index (0 .. L-1).
 //   v = fma(g, a, delta);  w = v + s;  k = clamp(rint(w), 0, L-1)   (clamping before rounding gives the same k)
-__device__ __forceinline__ float dqsg_index_f(float x, float a, float delta, const EncodeArgs& args)
+__device__ __forceinline__ uint32_t dqsg_index_bits(float x, float a, float delta, const EncodeArgs& args)
 {
     const float v = __fmaf_rn(x, a, delta);
     float w = __fadd_rn(v, args.shift);
     w = fminf(fmaxf(w, 0.0f), args.kmax);
-    return __fadd_rn(__fadd_rn(w, kMagic), -kMagic);                      // rint for 0 <= w < 2^22
+    return __float_as_uint(__fadd_rn(w, kMagic));                         // rint for 0 <= w < 2^22
 }
 
 // NDQSG: bit pattern kMagicBits + q1 (two's complement in the low bits) of one element.
@@ -115,66 +124,37 @@ __device__ __forceinline__ uint32_t ndqsg_index_bits(float x, float a, float del
 }
 
 // Quantize and pack one row.  x: the 32 elements; row: index of the row in the whole gradient (the Philox
-// counters follow from it; it differs from the row's position in this call's buffers when a bucket range is encoded); a: the bucket's gain.  out: the row's BITS words.  DITH: 32 or 16 random bits
-// per dither value.
+// counters follow from it; it differs from the row's position in this call's buffers when a bucket range is
+// encoded); a: the bucket's gain.  out: the row's BITS words.  DITH: 32 or 16 random bits per dither value.
 //
-// Integer and logic instructions cost about twice the issue bandwidth of fp32 ones on this GPU, so the DQSG
-// codes are packed in floating point: G = floor(22 / BITS) consecutive indices are combined by exact
-// multiply-adds (sum k_i 2^(BITS i) < 2^22) and only the group is converted and shifted into place.
-// NDQSG codes need their upper bits dropped; when BITS divides 32 that is one shift, and one funnel shift
-// inserts the code.
+// Adding 1.5 * 2^23 leaves the rounded index in the low mantissa bits of a float, so a code costs one fp32 add and
+// one funnel shift (push_code); only a coarse ratio below 2^BITS needs an extra mask or modulo.
 template <int BITS, int MODE, int DITH>
 __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, float a,
                                            const EncodeArgs& args, uint32_t (&out)[BITS])
 {
-#pragma unroll
-    for (int j = 0; j < BITS; ++j) out[j] = 0u;
-    constexpr int G = 22 / BITS;                    // elements per float group (DQSG)
     constexpr int EPB = (DITH == 16) ? 8 : 4;       // elements per Philox block
     constexpr int PASS = 4 * EPB;                   // elements per group of four blocks
-    float grp = 0.0f;
+    uint32_t sr = 0u;
 #pragma unroll
     for (int h = 0; h < 32 / PASS; ++h) {           // four Philox blocks in flight at a time
         uint32_t ctr[4], rnd[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) ctr[j] = row * (32u / EPB) + (uint32_t)(4 * h + j);
         philox4x32_10_xN<4>(ctr, args.ps, rnd);
-        if constexpr (MODE == kEncNdqsgPow2 && (32 % BITS) == 0) {
-            // K = 2^BITS here (the host sends any smaller power of two down the general path)
-            // units of U elements (a whole word, or half a word for one bit); elements are inserted from the
-            // last to the first: moving the code to the top of a register drops the bits above it, and one
-            // funnel shift pushes it into the unit.
-            constexpr int U = (32 / BITS < 16) ? (32 / BITS) : 16;
-            uint32_t unit = 0u;
 #pragma unroll
-            for (int t = PASS - 1; t >= 0; --t) {
-                const int idx = PASS * h + t;
-                const uint32_t tb = ndqsg_index_bits(x[idx], a, dither_delta_of<DITH>(rnd, t));
-                unit = __funnelshift_l(tb << (32 - BITS), (idx % U == U - 1) ? 0u : unit, BITS);
-                if (idx % U == 0) put_bits<BITS>(out, idx * BITS, U * BITS, unit);
+        for (int t = 0; t < PASS; ++t) {
+            const int idx = PASS * h + t;
+            const float delta = dither_delta_of<DITH>(rnd, t);
+            uint32_t tb;
+            if (MODE == kEncDqsg) {
+                tb = dqsg_index_bits(x[idx], a, delta, args);
+            } else {
+                tb = ndqsg_index_bits(x[idx], a, delta);
+                if (MODE == kEncNdqsgPow2Mask) tb &= args.K - 1u;
+                if (MODE == kEncNdqsgAnyK) tb = (tb - kMagicBits + args.K_offset) % args.K;   // q1 + positive multiple of K
             }
-        } else {
-#pragma unroll
-            for (int t = 0; t < PASS; ++t) {
-                const int idx = PASS * h + t;
-                const float delta = dither_delta_of<DITH>(rnd, t);
-                if (MODE == kEncDqsg) {
-                    const float kf = dqsg_index_f(x[idx], a, delta, args);
-                    const int pos = idx % G;                               // position inside the group
-                    grp = (pos == 0) ? kf : __fmaf_rn(kf, (float)(1u << (BITS * pos)), grp);   // exact
-                    if (pos == G - 1 || idx == 31) {
-                        const int first = idx - pos;
-                        const uint32_t gb = __float_as_uint(__fadd_rn(grp, kMagic)) - kMagicBits;
-                        put_bits<BITS>(out, first * BITS, (pos + 1) * BITS, gb);
-                    }
-                } else {
-                    const uint32_t tb = ndqsg_index_bits(x[idx], a, delta);
-                    uint32_t code;
-                    if (MODE == kEncNdqsgPow2) code = tb & (args.K - 1u);
-                    else code = (tb - kMagicBits + args.K_offset) % args.K;   // q1 + positive multiple of K
-                    put_bits<BITS>(out, idx * BITS, BITS, code);
-                }
-            }
+            push_code<BITS>(sr, tb, idx, out);
         }
     }
 }
@@ -400,8 +380,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         fence_mbar_init();
         asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmap) : "memory");
     }
-    // nothing above touches memory that an earlier kernel of the stream may still be writing
-    grid_dependency_wait();
+    // Nothing above touches memory that an earlier kernel of the stream may still be writing.  When the caller
+    // has declared the gradient complete (early_read), the tile copies and the arithmetic below only read memory
+    // that the previous kernel does not write, and the wait moves in front of this warp's first store.
+    bool waited = (args.early_read == 0u);
+    if (waited) grid_dependency_wait();
     if (lane == 0) {
         // All resident warps would request their first tiles (the whole shared memory of every SM, a quarter of a
         // ResNet-50-sized gradient) at the same instant; served interleaved, every warp would then get its data
@@ -450,7 +433,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                     if (!mbar_wait_bounded(my_bar, par, gave_up ? 1u : (1u << 22)) ||
                         !mbar_wait_bounded(my_bar + 8u, par, gave_up ? 1u : (1u << 22))) {
                         gave_up = true;
-                        if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
+                        if (lane == 0) atomicOr(args.error_flags, 0x2u);
                     }
                     // maximum of the second half, straight from shared memory
                     const uint32_t other = my_smem + kWarpTileBytes + lane * 128u;
@@ -485,7 +468,6 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                             if (i / wpb == group) mx = fmaxf(mx, o);
                         }
                     }
-                    if (lane == 0 && sub == 0u) args.scale[pair] = mx;
                 } else {
                     uint32_t sink = 0u;                 // all loads of this half have completed after this
 #pragma unroll
@@ -505,6 +487,8 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                 const uint32_t row = part * 64u + half * 32u + lane;
                 uint32_t out[BITS];
                 encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
+                if (!waited) { grid_dependency_wait(); waited = true; }
+                if (half == 0u && lane == 0 && sub == 0u) args.scale[pair] = mx;
                 store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
             }
         }
@@ -517,7 +501,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         const uint32_t use = k / kEncStages;
         if (!mbar_wait_bounded(my_bar + 8u * s, use & 1u, gave_up ? 1u : (1u << 22))) {
             gave_up = true;
-            if (lane == 0) atomicOr(&g_dq_error_flags, 0x2u);
+            if (lane == 0) atomicOr(args.error_flags, 0x2u);
         }
         // the lane's row -> registers
         float x[32];
@@ -549,11 +533,12 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
             }
         }
         const uint32_t row = (uint32_t)tile * 32u + lane;   // row index in the gradient (< 2^29)
-        if ((lane & (args.lanes_per_bucket - 1u)) == 0u) args.scale[row >> (args.bucket_log2 - 5u)] = mx;
         const float a = bucket_gain(args.gain_num, mx);
 
         uint32_t out[BITS];
         encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
+        if (!waited) { grid_dependency_wait(); waited = true; }
+        if ((lane & (args.lanes_per_bucket - 1u)) == 0u) args.scale[row >> (args.bucket_log2 - 5u)] = mx;
         store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
     }
 }
