@@ -1,6 +1,6 @@
 """Bandwidth sweep of the encode and fused decode-aggregate kernels (BASELINE config 5).
 
-    python -m paper_1904_01197_b200.sweep [--quick] [--out FILE]
+    python -m bench_tools.sweep [--quick] [--out FILE]
 
 Star design around (n = 2^26, W = 8, b = 2, B = 2048): one axis varies at a time; DQSG and NDQSG, both dither
 streams; each kernel is timed alone with CUDA events over buffers that rotate through more than 3x the L2 size
@@ -14,7 +14,7 @@ import json
 
 import torch
 
-from . import binding as dq
+from paper_1904_01197_b200 import binding as dq
 
 L2_BYTES = 126 * 1024 * 1024
 

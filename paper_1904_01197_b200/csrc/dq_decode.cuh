@@ -110,10 +110,8 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, co
     constexpr int PASS = 4 * EPB;                   // elements per group of four blocks
 #pragma unroll
     for (int h = 0; h < 32 / PASS; ++h) {
-        uint32_t ctr[4], rnd[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) ctr[j] = (uint32_t)row * (32u / EPB) + (uint32_t)(4 * h + j);
-        if (DITH != 0) philox4x32_10_xN<4>(ctr, wk.ps, rnd);
+        uint32_t rnd[4][4];
+        if (DITH != 0) philox4x32_10_row<4>((uint32_t)row * (32u / EPB), 4 * h, wk.ps, rnd);
 #pragma unroll
         for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};

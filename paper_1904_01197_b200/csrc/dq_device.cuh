@@ -29,6 +29,13 @@ struct PhiloxStream {
     uint32_t v3;          // lo(M0*u0) ^ rk[2][1]
 };
 
+// M0 * j for j = 0..7: the blocks of a row have consecutive counters base + j, and M0 * (base + j) is
+// M0 * base + M0 * j without a carry out of 64 bits, so the first multiply of block j takes its counter's offset
+// as the 64-bit addend of the multiply-add (an operand from constant memory) instead of an integer add of its own.
+static __constant__ uint64_t c_philox_m0j[8] = {
+    0ull * kPhiloxM0, 1ull * kPhiloxM0, 2ull * kPhiloxM0, 3ull * kPhiloxM0,
+    4ull * kPhiloxM0, 5ull * kPhiloxM0, 6ull * kPhiloxM0, 7ull * kPhiloxM0};
+
 // N blocks at once, rounds outermost, so N independent dependency chains are in flight.
 // Counter word 0 of block j is c0[j] = index of its 4-element chunk (element index / 4).
 template <int N>
@@ -52,6 +59,51 @@ __device__ __forceinline__ void philox4x32_10_xN(const uint32_t (&c0in)[N], cons
         c2[j] = c3[j] ^ ps.v2;
     }
     // round 2: c3 is block-independent (folded into v3)
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0[j];
+        const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2[j];
+        c0[j] = (uint32_t)(p1 >> 32) ^ c1[j] ^ ps.rk[2][0];
+        c1[j] = (uint32_t)p1;
+        c2[j] = (uint32_t)(p0 >> 32) ^ ps.v3;
+        c3[j] = (uint32_t)p0;
+    }
+#pragma unroll
+    for (int r = 3; r < 10; ++r) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0[j];
+            const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2[j];
+            c0[j] = (uint32_t)(p1 >> 32) ^ c1[j] ^ ps.rk[r][0];
+            c1[j] = (uint32_t)p1;
+            c2[j] = (uint32_t)(p0 >> 32) ^ c3[j] ^ ps.rk[r][1];
+            c3[j] = (uint32_t)p0;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < N; ++j) { out[j][0] = c0[j]; out[j][1] = c1[j]; out[j][2] = c2[j]; out[j][3] = c3[j]; }
+}
+
+// The same for the N consecutive blocks base + first, ..., base + first + N - 1 of a row (first + N <= 8 and
+// base + 7 < 2^32): see c_philox_m0j.
+template <int N>
+__device__ __forceinline__ void philox4x32_10_row(uint32_t base, int first, const PhiloxStream& ps,
+                                                  uint32_t (&out)[N][4])
+{
+    uint32_t c0[N], c1[N], c2[N], c3[N];
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)base + c_philox_m0j[first + j];
+        c2[j] = (uint32_t)(p0 >> 32) ^ ps.v0;
+        c3[j] = (uint32_t)p0;
+    }
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+        const uint64_t p1 = (uint64_t)kPhiloxM1 * (uint64_t)c2[j];
+        c0[j] = (uint32_t)(p1 >> 32) ^ ps.v1;
+        c1[j] = (uint32_t)p1;
+        c2[j] = c3[j] ^ ps.v2;
+    }
 #pragma unroll
     for (int j = 0; j < N; ++j) {
         const uint64_t p0 = (uint64_t)kPhiloxM0 * (uint64_t)c0[j];

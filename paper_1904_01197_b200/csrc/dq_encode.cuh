@@ -138,10 +138,8 @@ __device__ __forceinline__ void encode_row(const float (&x)[32], uint32_t row, f
     uint32_t sr = 0u;
 #pragma unroll
     for (int h = 0; h < 32 / PASS; ++h) {           // four Philox blocks in flight at a time
-        uint32_t ctr[4], rnd[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) ctr[j] = row * (32u / EPB) + (uint32_t)(4 * h + j);
-        philox4x32_10_xN<4>(ctr, args.ps, rnd);
+        uint32_t rnd[4][4];
+        philox4x32_10_row<4>(row * (32u / EPB), 4 * h, args.ps, rnd);
 #pragma unroll
         for (int t = 0; t < PASS; ++t) {
             const int idx = PASS * h + t;
@@ -409,7 +407,10 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     }
     __syncwarp();
 
-    const uint32_t swz = lane & 7u;                  // (row & 7): the warp's rows start at a multiple of 32
+    // 128-byte swizzle: the 16-byte piece c of row r sits at piece c ^ (r & 7).  A lane's row starts at a multiple
+    // of 128 bytes, so "row address + ((c ^ swz) << 4)" is "(row address | swz << 4) ^ (c << 4)": one XOR with
+    // an immediate per load.
+    const uint32_t swz16 = (lane & 7u) << 4;         // (row & 7) << 4: the warp's rows start at a multiple of 32
     bool gave_up = false;
     uint32_t k = 0;
 
@@ -428,7 +429,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
             float mx = 0.0f;
 #pragma unroll 1
             for (uint32_t half = 0; half < 2u; ++half) {
-                const uint32_t stage_addr = my_smem + half * kWarpTileBytes + lane * 128u;
+                const uint32_t stage_addr = (my_smem + half * kWarpTileBytes + lane * 128u) | swz16;
                 if (half == 0u) {
                     if (!mbar_wait_bounded(my_bar, par, gave_up ? 1u : (1u << 22)) ||
                         !mbar_wait_bounded(my_bar + 8u, par, gave_up ? 1u : (1u << 22))) {
@@ -436,13 +437,13 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                         if (lane == 0) atomicOr(args.error_flags, 0x2u);
                     }
                     // maximum of the second half, straight from shared memory
-                    const uint32_t other = my_smem + kWarpTileBytes + lane * 128u;
+                    const uint32_t other = (my_smem + kWarpTileBytes + lane * 128u) | swz16;
 #pragma unroll
                     for (uint32_t c = 0; c < 8; ++c) {
                         float4 v;
                         asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
                                      : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                                     : "r"(other + ((c ^ swz) << 4))
+                                     : "r"(other ^ (c << 4))
                                      : "memory");
                         mx = max3_abs(max3_abs(mx, v.x, v.y), v.z, v.w);
                     }
@@ -451,7 +452,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                 for (uint32_t c = 0; c < 8; ++c) {
                     asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
                                  : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
-                                 : "r"(stage_addr + ((c ^ swz) << 4))
+                                 : "r"(stage_addr ^ (c << 4))
                                  : "memory");
                 }
                 if (half == 0u) {
@@ -505,12 +506,12 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
         }
         // the lane's row -> registers
         float x[32];
-        const uint32_t row_addr = my_smem + s * kWarpTileBytes + lane * 128u;
+        const uint32_t row_addr = (my_smem + s * kWarpTileBytes + lane * 128u) | swz16;
 #pragma unroll
         for (uint32_t c = 0; c < 8; ++c) {
             asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
                          : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
-                         : "r"(row_addr + ((c ^ swz) << 4))
+                         : "r"(row_addr ^ (c << 4))
                          : "memory");
         }
         // max |g| over the bucket.  Every lane has used all of its loaded values once it reaches the
