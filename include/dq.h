@@ -80,6 +80,15 @@ typedef struct {
  * complete, so outputs may be shared with it.  Results are identical with and without the flag.
  */
 #define DQ_FLAG_INPUT_READY 0x1u
+/*
+ * DQ_FLAG_OUTPUT_FREE (encoders only; has an effect only together with DQ_FLAG_INPUT_READY).  The caller
+ * additionally declares that the previous kernel of the stream neither reads nor writes out_packed and
+ * out_scale -- e.g. the encodes of different workers' gradients into different message buffers, back to back.
+ * Then nothing in the encoder waits for that kernel except its own end: the two kernels overlap wherever the
+ * GPU has room (the tail of one runs beside the head of the next), while a later kernel that waits for this
+ * one still sees both complete.  Results are identical with and without the flag.
+ */
+#define DQ_FLAG_OUTPUT_FREE 0x2u
 
 /* One worker's message as the decoder sees it. */
 typedef struct {

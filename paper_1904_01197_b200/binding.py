@@ -19,6 +19,7 @@ DQ_WARN_NONFINITE_SCALE = 0x1
 DQ_ERR_COPY_TIMEOUT = 0x2
 DQ_WARN_CODE_RANGE = 0x4
 DQ_FLAG_INPUT_READY = 0x1
+DQ_FLAG_OUTPUT_FREE = 0x2
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libdq_b200.so"
 

@@ -57,10 +57,10 @@ def stale() -> bool:
     return any(d.stat().st_mtime > t for d in DEPS)
 
 
-def _compile(unit, verbose: bool) -> Path:
+def _compile(unit, verbose: bool, obj_dir: Path = OBJ, extra_flags=()) -> Path:
     name, src, defs = unit
-    obj = OBJ / f"{name}.o"
-    cmd = [nvcc_path(), *NVCC_FLAGS, *defs, f"-I{ROOT / 'include'}", f"-I{CSRC}", "-c", "-o", str(obj),
+    obj = obj_dir / f"{name}.o"
+    cmd = [nvcc_path(), *NVCC_FLAGS, *defs, *extra_flags, f"-I{ROOT / 'include'}", f"-I{CSRC}", "-c", "-o", str(obj),
            str(CSRC / src)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
@@ -68,18 +68,28 @@ def _compile(unit, verbose: bool) -> Path:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
+def build(force: bool = False, verbose: bool = False, out: Path | None = None, extra_flags=()) -> Path:
+    """Compiles every translation unit and links the shared library.  `out` / `extra_flags` build a variant
+    (other tile or occupancy constants, see the DQ_* macros in csrc/) beside the default library."""
+    if out is not None:
+        return _build_to(Path(out), list(extra_flags), verbose)
     if not force and not stale():
         return LIB
-    OBJ.mkdir(parents=True, exist_ok=True)
+    return _build_to(LIB, [], verbose)
+
+
+def _build_to(lib: Path, extra_flags, verbose: bool) -> Path:
+    global OBJ
+    obj_dir = OBJ if lib == LIB else lib.parent / (lib.stem + "_obj")
+    obj_dir.mkdir(parents=True, exist_ok=True)
     jobs = int(os.environ.get("DQ_BUILD_JOBS", "0")) or min(len(UNITS), os.cpu_count() or 1)
     with ThreadPoolExecutor(max_workers=jobs) as pool:
-        objs = list(pool.map(lambda u: _compile(u, verbose), UNITS))
-    tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
+        objs = list(pool.map(lambda u: _compile(u, verbose, obj_dir, extra_flags), UNITS))
+    tmp = lib.with_suffix(f".{os.getpid()}.tmp")
     subprocess.run([nvcc_path(), "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
                     "-o", str(tmp), *[str(o) for o in objs]], check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

@@ -205,6 +205,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     }
     fill_philox(a.ps, seed, worker, step);
     a.early_read = (p->flags & DQ_FLAG_INPUT_READY) ? 1u : 0u;
+    a.early_store = (a.early_read && (p->flags & DQ_FLAG_OUTPUT_FREE)) ? 1u : 0u;
     a.error_flags = error_flags_address();
     if (!a.error_flags) return DQ_ERR_CUDA;
 

@@ -79,6 +79,8 @@ struct EncodeArgs {
     uint32_t early_read;     // the caller guarantees that grad was complete before the previous kernel of the stream
                              // began: the tile path requests (and quantizes) its first tiles while that kernel
                              // drains, and only its stores wait for it
+    uint32_t early_store;    // ... and that the previous kernel neither reads nor writes this call's outputs: nothing
+                             // waits for that kernel except the end of this one (see encode_kernel)
     unsigned int* error_flags;     // the library's per-device error word
     PhiloxStream ps;
 };
@@ -380,8 +382,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     }
     // Nothing above touches memory that an earlier kernel of the stream may still be writing.  When the caller
     // has declared the gradient complete (early_read), the tile copies and the arithmetic below only read memory
-    // that the previous kernel does not write, and the wait moves in front of this warp's first store.
+    // that the previous kernel does not write, and the wait moves in front of this warp's first store; when the
+    // outputs are declared free as well (early_store), it moves to the end of the warp's work, where it only keeps
+    // this grid from completing before its predecessor (a later kernel that waits for this one may rely on both).
     bool waited = (args.early_read == 0u);
+    const bool wait_before_store = (args.early_store == 0u);
     if (waited) grid_dependency_wait();
     if (lane == 0) {
         // All resident warps would request their first tiles (the whole shared memory of every SM, a quarter of a
@@ -488,11 +493,12 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                 const uint32_t row = part * 64u + half * 32u + lane;
                 uint32_t out[BITS];
                 encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
-                if (!waited) { grid_dependency_wait(); waited = true; }
+                if (!waited && wait_before_store) { grid_dependency_wait(); waited = true; }
                 if (half == 0u && lane == 0 && sub == 0u) args.scale[pair] = mx;
                 store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
             }
         }
+        if (!waited) grid_dependency_wait();
         return;
     }
 
@@ -538,10 +544,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
 
         uint32_t out[BITS];
         encode_row<BITS, MODE, DITH>(x, row + args.row_offset, a, args, out);
-        if (!waited) { grid_dependency_wait(); waited = true; }
+        if (!waited && wait_before_store) { grid_dependency_wait(); waited = true; }
         if ((lane & (args.lanes_per_bucket - 1u)) == 0u) args.scale[row >> (args.bucket_log2 - 5u)] = mx;
         store_row_words<BITS>(args.packed + (uint64_t)row * BITS, out);
     }
+    if (!waited) grid_dependency_wait();
 }
 
 }  // namespace dq
