@@ -32,6 +32,12 @@ T* virtual_base(T* p, uint64_t first)
 {
     return reinterpret_cast<T*>(reinterpret_cast<uintptr_t>(p) - first * sizeof(T));
 }
+bool float_is_pow2(float v)
+{
+    uint32_t u;
+    std::memcpy(&u, &v, sizeof(u));
+    return v > 0.0f && (u & 0x007FFFFFu) == 0u && (u >> 23) != 0u && (u >> 23) != 0xFFu;
+}
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0u; }
 
 void fill_philox(dq::PhiloxStream& ps, uint64_t seed, uint32_t worker, uint64_t step)
@@ -116,7 +122,7 @@ encode_tiled_fn get_encode_tiled()
 }
 
 // [rows x 32 fp32] view of a flat vector, boxes of `box_rows` rows, 128-byte swizzle.
-bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t box_rows)
+bool make_row_map(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows)
 {
     encode_tiled_fn fn = get_encode_tiled();
     if (!fn) return false;
@@ -124,7 +130,7 @@ bool make_row_map(CUtensorMap* map, const float* base, uint64_t rows, uint32_t b
     const cuuint64_t strides[1] = {128u};
     const cuuint32_t box[2] = {32u, box_rows};
     const cuuint32_t estr[2] = {1u, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2u, const_cast<float*>(base), dims, strides, box, estr,
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2u, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -290,16 +296,19 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         // addresses of the (virtual) whole-gradient buffers: see DecodeArgs
         d.packed = virtual_base(m.packed, first_element / 32u * m.p.bits);
         d.scale = virtual_base(m.scale, first_element / m.p.bucket);
+        d.unit_lines = m.p.bits;
         fill_philox(d.ps, m.seed, m.worker, step);
         d.bits = m.p.bits;
+        uint32_t kind;
         if (m.kind == DQ_KIND_DQSG) {
-            d.kind = dq::kDecDqsg;
+            kind = dq::kDecDqsg;
             d.s = (float)(L - 1u) / 2.0f;
             d.cconst = 4194304.0f + d.s - 1.5f;
+            d.step_mul = is_pow2(L - 1u) && L >= 3u ? 2.0f / (float)(L - 1u) : (L == 2u ? 2.0f : 0.0f);
         } else {
             any_nested = true;
-            if (!is_pow2(m.p.coarse_K)) d.kind = dq::kDecNdqsgAnyK;
-            else d.kind = (alpha == 1.0f) ? dq::kDecNdqsgPow2 : dq::kDecNdqsgPow2Shrink;
+            if (!is_pow2(m.p.coarse_K)) kind = dq::kDecNdqsgAnyK;
+            else kind = (alpha == 1.0f) ? dq::kDecNdqsgPow2 : dq::kDecNdqsgPow2Shrink;
             d.cconst = 4194304.0f - 1.5f;
             d.A = alpha * m.p.fine_M;
             d.M1 = m.p.fine_M;
@@ -308,11 +317,13 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
             d.one_m_alpha2 = 1.0f - a2;
             d.Kf = (float)m.p.coarse_K;
             d.invK = 1.0f / d.Kf;
+            d.step_mul = float_is_pow2(m.p.fine_M) ? 1.0f / m.p.fine_M : 0.0f;
             if (running) {
                 if (w == 0u) return DQ_ERR_INVALID_ARG;      // nothing decoded yet to serve as side information
                 d.rcp_count = 1.0f / (float)w;
             }
         }
+        d.variant = kind * 8u + m.p.bits - 1u;
     }
     if (first_element % msgs[0].p.bucket != 0u) return DQ_ERR_INVALID_ARG;   // a range starts at a bucket boundary
     if (n == 0) return DQ_OK;
@@ -325,30 +336,47 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
         if (!aligned16(msgs[w].packed) || !aligned16(msgs[w].scale)) return DQ_ERR_ALIGNMENT;
     }
-    a.side = (any_nested && !running) ? virtual_base(side_info, first_element) : nullptr;
+    const bool reads_side = any_nested && !running;
+    a.side = reads_side ? virtual_base(side_info, first_element) : nullptr;
     a.out = virtual_base(out_avg, first_element);
     a.status = status_word;
     a.n = first_element + n;
-    a.rows = (first_element + n + 31u) / 32u;
-    a.first_row = first_element / 32u;
-    {
-        const int sms_now = device_sm_count();
-        // one block per SM ahead: 16 to 200 blocks measured alike, a whole wave (4 per SM) or more is too far
-        a.prefetch_blocks = (sms_now > 0) ? (uint32_t)sms_now : 0u;
-    }
+    a.rows = (uint32_t)((first_element + n + 31u) / 32u);
+    a.first_row = (uint32_t)(first_element / 32u);
+    a.full_rows = (uint32_t)((first_element + n) / 32u);
+    a.num_units = (a.rows - a.first_row + 31u) / 32u;
     a.W = W;
     a.rows_per_bucket = msgs[0].p.bucket / 32u;
+    a.rpb_shift = 0xFFFFFFFFu;
+    if (is_pow2(a.rows_per_bucket)) {
+        a.rpb_shift = 0u;
+        while ((1u << a.rpb_shift) < a.rows_per_bucket) ++a.rpb_shift;
+    }
+    a.has_side = reads_side ? 1u : 0u;
     a.half_bias_bits = 0x4A800000u;
     a.Wf = (float)W;
     a.invW = is_pow2(W) ? 1.0f / (float)W : 0.0f;
-    const uint64_t grid64 = (a.rows - a.first_row + dq::kDecThreads - 1u) / dq::kDecThreads;
-    if (grid64 > 0x7FFFFFFFull) return DQ_ERR_UNSUPPORTED;
+    a.error_flags = error_flags_address();
+    if (!a.error_flags) return DQ_ERR_CUDA;
+    // tile views of the caller's buffers: whole rows only (a ragged last row is handled with plain accesses)
+    CUtensorMap side_map, out_map;
+    std::memset(&side_map, 0, sizeof(side_map));
+    std::memset(&out_map, 0, sizeof(out_map));
+    const uint32_t whole_rows = a.full_rows - a.first_row;
+    a.use_tiles = whole_rows != 0u ? 1u : 0u;
+    if (whole_rows != 0u) {
+        if (!make_row_map(&out_map, out_avg, whole_rows, 32u)) return DQ_ERR_CUDA;
+        if (reads_side && !make_row_map(&side_map, side_info, whole_rows, 32u)) return DQ_ERR_CUDA;
+    }
+    const int sms = device_sm_count();
+    if (sms <= 0) return DQ_ERR_CUDA;
     const bool d16 = (msgs[0].p.dither_bits == 16u);
-    const uint32_t grid = (uint32_t)grid64;
     cudaError_t le;
-    if (half_dithered) le = dq::launch_decode_d0_r0(a, grid, st);
-    else if (running && any_nested) le = d16 ? dq::launch_decode_d16_r1(a, grid, st) : dq::launch_decode_d32_r1(a, grid, st);
-    else le = d16 ? dq::launch_decode_d16_r0(a, grid, st) : dq::launch_decode_d32_r0(a, grid, st);
+    if (half_dithered) le = dq::launch_decode_d0_r0(side_map, out_map, a, sms, st);
+    else if (running && any_nested) le = d16 ? dq::launch_decode_d16_r1(side_map, out_map, a, sms, st)
+                                             : dq::launch_decode_d32_r1(side_map, out_map, a, sms, st);
+    else le = d16 ? dq::launch_decode_d16_r0(side_map, out_map, a, sms, st)
+                  : dq::launch_decode_d32_r0(side_map, out_map, a, sms, st);
     if (le != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);
     return DQ_OK;

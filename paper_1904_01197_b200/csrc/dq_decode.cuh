@@ -1,15 +1,23 @@
 // Fused decode-and-average kernel (Algorithm 1, server steps; nested decoder equation and Algorithm 2,
 // server loop with the side information given as a vector or taken as the running mean).
 //
-// One lane owns one row = 32 consecutive elements: 32 fp32 accumulators in registers, and per worker
-// exactly `bits` packed words.  For every worker (in array order) the lane reloads that worker's words and
-// bucket scale, regenerates the 32 dithers (Philox blocks four at a time, so four dependency chains are in
-// flight), reconstructs and accumulates; the mean is written at the end.  The packed streams, the side
-// information and the output are each touched once in HBM (the side information of a CTA's 128 rows is staged
-// in swizzled shared memory and re-read from there per worker, which keeps it out of the register file).
+// One lane owns one row = 32 consecutive elements: 32 fp32 accumulators in registers, and per worker exactly
+// `bits` packed words.  A warp owns a unit of 32 rows and is autonomous: persistent warps take units round-robin
+// and never wait for one another.
+//   * The side information of a unit arrives in the warp's shared memory by one 2-D tile copy (32 rows x 128
+//     bytes, 128-byte swizzle, so that "lane r reads row r" is free of bank conflicts), issued one unit ahead.
+//   * Every worker's packed words of the next unit are requested into the L2 one unit ahead (one prefetch
+//     instruction per unit: lane w asks for worker w's lines); each lane then loads exactly its `bits` words with
+//     the widest vector loads their alignment allows, and the Philox work that follows hides the L2 latency.
+//   * For every worker (in array order) the lane regenerates the 32 dithers (Philox blocks four at a time),
+//     reconstructs and accumulates; the bucket scale is loaded one step ahead.
+//   * The mean goes back through the tile buffer and leaves with one tile store per unit: full 128-byte lines,
+//     issued by one lane.
+// The packed streams, the side information and the output are each touched once in HBM.
 //
 // The path is bound by instruction issue, not by HBM: each (element, worker) pair needs a quarter of a
-// Philox block (9.25 integer instructions) before any reconstruction arithmetic.
+// Philox block (4.5 wide multiplies, which occupy the multiplier pipe for four cycles each) before any
+// reconstruction arithmetic.
 #pragma once
 
 #include "dq_device.cuh"
@@ -19,10 +27,11 @@ namespace dq {
 enum DecKind : uint32_t { kDecDqsg = 0, kDecNdqsgPow2 = 1, kDecNdqsgPow2Shrink = 2, kDecNdqsgAnyK = 3 };
 
 struct DecWorker {
-    const uint32_t* packed;
-    const float* scale;
+    const uint32_t* packed;   // } addresses of the (virtual) whole-gradient buffers, see DecodeArgs
+    const float* scale;       // }
+    uint32_t unit_lines;      // 128-byte lines of one unit's packed words (= bits)
     PhiloxStream ps;
-    uint32_t kind;        // DecKind
+    uint32_t variant;     // DecKind * 8 + bits - 1: one jump selects the routine
     uint32_t bits;
     float s;              // DQSG (L-1)/2
     float cconst;         // DQSG: 4194304 + s - 1.5 ; NDQSG: 4194304 - 1.5   (see unpack_half_biased)
@@ -33,6 +42,8 @@ struct DecWorker {
     float Kf;             // (float)K
     float invK;           // 1/K (exact when K is a power of two)
     float rcp_count;      // running-mean mode: 1 / (number of workers before this one)
+    float step_mul;       // DQSG: 1/s, NDQSG: 1/M1, when that divisor is a power of two (the division is then an
+                          // exact multiplication); 0 otherwise
 };
 
 struct DecodeArgs {
@@ -41,23 +52,39 @@ struct DecodeArgs {
     uint32_t* status;
     // A call may cover the elements [first, n) of a longer gradient (first a multiple of the bucket size, 0 for a
     // whole gradient).  Rows, elements and buckets are then numbered as in the whole gradient -- which is what the
-    // dither counters need -- and every pointer below is the buffer's address minus the range's offset, so that
-    // "pointer + global index" lands in the caller's buffer.
+    // dither counters need -- and every pointer above and in w[] is the buffer's address minus the range's offset,
+    // so that "pointer + global index" lands in the caller's buffer.  The tile maps cover the caller's buffers
+    // themselves (row 0 of a map = row first_row of the gradient) and only whole rows.
     uint64_t n;               // end of the range (element index)
-    uint64_t rows;            // ceil(n / 32): end of the range (row index)
-    uint64_t first_row;       // first / 32
-    uint32_t prefetch_blocks; // distance, in 128-row blocks, of the L2 prefetch (0 = none)
+    uint32_t rows;            // ceil(n / 32): end of the range (row index); below 2^29
+    uint32_t first_row;       // first / 32
+    uint32_t full_rows;       // floor(n / 32): rows below this index have 32 elements
+    uint32_t num_units;       // ceil((rows - first_row) / 32): units of 32 rows
     uint32_t W;
     uint32_t rows_per_bucket; // B / 32
+    uint32_t rpb_shift;       // log2(rows_per_bucket) when that is a power of two, else 0xFFFFFFFF
+    uint32_t has_side;        // the side information vector is read (some message is NDQSG, not running-mean mode)
+    uint32_t use_tiles;       // the range holds at least one whole row: the tile maps are valid
     uint32_t half_bias_bits;  // 0x4A800000 (bit pattern of 2^22), passed in so that it lives in a register
     float Wf;
     float invW;               // 1/W when W is a power of two, else 0
+    unsigned int* error_flags;    // the library's per-device error word
     DecWorker w[64];
 };
 
-// Code of element `idx` of a row, returned as the float 2^22 + code/1 ... precisely: the bit pattern of
-// 2^22 with the code in mantissa bits 1.., i.e. the value 2^22 + code (floats in [2^22, 2^23) step by 1/2).
-// Subtracting a constant then gives code - c exactly.
+constexpr int kDecThreads = 128;
+constexpr int kDecWarps = kDecThreads / 32;
+#ifndef DQ_DEC_MINBLOCKS
+#define DQ_DEC_MINBLOCKS 4
+#endif
+constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;     // resident CTAs per SM the register budget is set for
+constexpr int kDecTileBytes = 32 * 128;         // one unit of side information or output
+constexpr int kDecTileBuffers = 3;              // per warp: side in flight / side in use, then output leaving
+// Dynamic shared memory of a CTA: the warps' tile buffers (plus room to align to 1024 bytes).
+constexpr uint32_t kDecSmemBytes = (uint32_t)(kDecWarps * kDecTileBuffers * kDecTileBytes) + 1024u;
+
+// Code of element `idx` of a row as the float 2^22 + code: the bit pattern of 2^22 with the code in mantissa
+// bits 1.. (floats in [2^22, 2^23) step by 1/2).  Subtracting a constant then gives code - c exactly.
 template <int BITS>
 __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS], int idx, uint32_t bias_bits)
 {
@@ -74,52 +101,65 @@ __device__ __forceinline__ float unpack_half_biased(const uint32_t (&words)[BITS
     return __uint_as_float((v & mask2) | bias_bits);          // one logic op: (v & immediate) | register
 }
 
-// A worker's packed words of one row (bits words, at most 8) and its bucket scale.
-__device__ __forceinline__ void load_worker_row(const DecWorker& wk, uint64_t row, uint64_t bucket,
-                                                uint32_t (&words)[8], float& kappa)
+// The lane's BITS words (p = address of the first one; a row of BITS words starts at a multiple of 4 * BITS
+// bytes), with the widest loads that alignment allows.
+template <int BITS>
+__device__ __forceinline__ void load_words(const uint32_t* p, uint32_t (&w)[BITS])
 {
-    const uint32_t* src = wk.packed + row * wk.bits;
+    if constexpr (BITS % 4 == 0) {
 #pragma unroll
-    for (uint32_t j = 0; j < 8; ++j)
-        if (j < wk.bits) words[j] = __ldg(src + j);
-    kappa = __ldg(wk.scale + bucket);
+        for (int j = 0; j < BITS; j += 4) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p + j));
+            w[j] = v.x; w[j + 1] = v.y; w[j + 2] = v.z; w[j + 3] = v.w;
+        }
+    } else if constexpr (BITS % 2 == 0) {
+#pragma unroll
+        for (int j = 0; j < BITS; j += 2) {
+            const uint2 v = __ldg(reinterpret_cast<const uint2*>(p + j));
+            w[j] = v.x; w[j + 1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < BITS; ++j) w[j] = __ldg(p + j);
+    }
 }
 
 // One worker's contribution to the 32 accumulators of a row.
 //   DQSG:  g~ = (kappa/s) ((k - s) - delta); (k - s + 1.5) - f rounds once to the same value.
 //   NDQSG: r = (m - delta) - y a;  jj = rint(r / K);  q1^ = m - K jj;  g~ = beta (q1^ - delta) [+ (1-alpha^2) y]
+// load_row: the row whose words the lane loads (its own row, or the last whole row for lanes past the end, whose
+// results are never stored); side_addr: shared-memory address of
+// the lane's row of side information with the swizzle term already OR-ed in (piece p is at side_addr ^ (p << 4)).
 template <int BITS, uint32_t KIND, int DITH, bool RUN>
-__device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, const uint32_t (&cur)[8],
-                                           float kappa, const float* side_row, float (&acc)[32],
-                                           uint32_t* status, uint32_t bias_bits)
+__device__ __forceinline__ void decode_row(const DecWorker& wk, uint32_t row, uint32_t load_row, float kappa,
+                                           uint32_t side_addr, float (&acc)[32], uint32_t bias_bits)
 {
     uint32_t words[BITS];
-#pragma unroll
-    for (int j = 0; j < BITS; ++j) words[j] = cur[j];
+    load_words<BITS>(wk.packed + (uint64_t)load_row * (uint32_t)BITS, words);
 
-    if (status != nullptr && !(fabsf(kappa) <= 3.402823466e38f)) atomicOr(status, 0x1u);
-
+    // kappa / s and alpha kappa / M1: a division by a power of two is an exact multiplication
     float c, a = 0.0f;
     if (KIND == kDecDqsg) {
-        c = __fdiv_rn(kappa, wk.s);
+        c = (wk.step_mul != 0.0f) ? __fmul_rn(kappa, wk.step_mul) : __fdiv_rn(kappa, wk.s);
     } else {
         a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
-        c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);                 // beta
+        const float ak = __fmul_rn(wk.alpha, kappa);
+        c = (wk.step_mul != 0.0f) ? __fmul_rn(ak, wk.step_mul) : __fdiv_rn(ak, wk.M1);            // beta
     }
     constexpr int EPB = (DITH == 16) ? 8 : 4;       // elements per Philox block
     constexpr int PASS = 4 * EPB;                   // elements per group of four blocks
 #pragma unroll
     for (int h = 0; h < 32 / PASS; ++h) {
         uint32_t rnd[4][4];
-        if (DITH != 0) philox4x32_10_row<4>((uint32_t)row * (32u / EPB), 4 * h, wk.ps, rnd);
+        if (DITH != 0) philox4x32_10_row<4>(row * (32u / EPB), 4 * h, wk.ps, rnd);
 #pragma unroll
         for (int q = 0; q < PASS / 4; ++q) {        // four elements at a time (one 16-byte piece of y)
             float y[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (KIND != kDecDqsg && !RUN) {
-                // the row's side information sits in shared memory, 16-byte pieces swizzled by (row & 7)
-                const uint32_t piece = (uint32_t)((PASS / 4) * h + q) ^ (threadIdx.x & 7u);
-                const float4 v = *reinterpret_cast<const float4*>(side_row + 4u * piece);
-                y[0] = v.x; y[1] = v.y; y[2] = v.z; y[3] = v.w;
+                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                             : "=f"(y[0]), "=f"(y[1]), "=f"(y[2]), "=f"(y[3])
+                             : "r"(side_addr ^ (uint32_t)(((PASS / 4) * h + q) << 4))
+                             : "memory");
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -157,34 +197,42 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint64_t row, co
     }
 }
 
-template <uint32_t KIND, int DITH, bool RUN>
-__device__ __forceinline__ void decode_row_bits(const DecWorker& wk, uint64_t row, const uint32_t (&cur)[8],
-                                                float kappa, const float* side_row, float (&acc)[32],
-                                                uint32_t* status, uint32_t bias_bits)
+// Dispatch on (kind, bits): one indexed jump.
+template <int DITH, bool RUN>
+__device__ __forceinline__ void decode_row_variant(const DecWorker& wk, uint32_t row, uint32_t load_row,
+                                                   float kappa, uint32_t side_addr, float (&acc)[32],
+                                                   uint32_t bias_bits)
 {
-    switch (wk.bits) {
-        case 1: decode_row<1, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        case 2: decode_row<2, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        case 3: decode_row<3, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        case 4: decode_row<4, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        case 5: decode_row<5, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        case 6: decode_row<6, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        case 7: decode_row<7, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
-        default: decode_row<8, KIND, DITH, RUN>(wk, row, cur, kappa, side_row, acc, status, bias_bits); break;
+#define DQ_DEC_CASE(KIND, BITS)                                                                                    \
+    case (KIND) * 8u + (BITS) - 1u:                                                                                \
+        decode_row<BITS, KIND, DITH, RUN>(wk, row, load_row, kappa, side_addr, acc, bias_bits);                        \
+        break;
+#define DQ_DEC_KIND(KIND)                                                                                          \
+    DQ_DEC_CASE(KIND, 1) DQ_DEC_CASE(KIND, 2) DQ_DEC_CASE(KIND, 3) DQ_DEC_CASE(KIND, 4)                            \
+    DQ_DEC_CASE(KIND, 5) DQ_DEC_CASE(KIND, 6) DQ_DEC_CASE(KIND, 7) DQ_DEC_CASE(KIND, 8)
+    switch (wk.variant) {
+        DQ_DEC_KIND(kDecDqsg)
+        DQ_DEC_KIND(kDecNdqsgPow2)
+        DQ_DEC_KIND(kDecNdqsgPow2Shrink)
+        DQ_DEC_KIND(kDecNdqsgAnyK)
+        default: break;
     }
+#undef DQ_DEC_KIND
+#undef DQ_DEC_CASE
 }
 
 // The last row of a gradient whose length is not a multiple of 32: one element at a time, everything at run
-// time.  Same arithmetic, in the same order, as decode_row.
+// time, straight from and to global memory.  Same arithmetic, in the same order, as decode_row.
 template <int DITH, bool RUN>
-__device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t row, uint64_t bucket, uint32_t nvalid)
+__device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint32_t row, uint32_t bucket, uint32_t nvalid)
 {
     for (uint32_t e = 0; e < nvalid; ++e) {
-        const uint64_t i = row * 32u + e;
-        const float yside = (!RUN && args.side) ? __ldg(args.side + i) : 0.0f;
+        const uint64_t i = (uint64_t)row * 32u + e;
+        const float yside = (!RUN && args.has_side) ? __ldg(args.side + i) : 0.0f;
         float acc = 0.0f;
         for (uint32_t w = 0; w < args.W; ++w) {
             const DecWorker& wk = args.w[w];
+            const uint32_t kind = wk.variant >> 3;
             const uint32_t bits = wk.bits;
             const uint64_t bit = i * bits;
             const uint64_t num_words = (args.n * bits + 31u) >> 5;
@@ -210,14 +258,14 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t
             if (args.status != nullptr && !(fabsf(kappa) <= 3.402823466e38f)) atomicOr(args.status, 0x1u);
             const float X = __fadd_rn(__uint_as_float((code << 1) | 0x4A800000u), -wk.cconst);
             float gt;
-            if (wk.kind == kDecDqsg) {
+            if (kind == kDecDqsg) {
                 gt = __fmul_rn(__fdiv_rn(kappa, wk.s), __fadd_rn(X, -f));
             } else {
                 const float yy = RUN ? __fmul_rn(acc, wk.rcp_count) : yside;
                 const float a = (kappa >= 0x1p-100f) ? __fdiv_rn(wk.A, kappa) : 0.0f;
                 const float c = __fdiv_rn(__fmul_rn(wk.alpha, kappa), wk.M1);
                 const float r = __fmaf_rn(-yy, a, __fadd_rn(X, -f));
-                const float t = (wk.kind == kDecNdqsgAnyK) ? __fdiv_rn(r, wk.Kf) : __fmul_rn(r, wk.invK);
+                const float t = (kind == kDecNdqsgAnyK) ? __fdiv_rn(r, wk.Kf) : __fmul_rn(r, wk.invK);
                 const float jj = __fadd_rn(__fadd_rn(t, kMagic), -kMagic);
                 const float d = __fadd_rn(__fmaf_rn(-wk.Kf, jj, X), -f);
                 gt = (wk.alpha == 1.0f) ? __fmul_rn(c, d) : __fmaf_rn(c, d, __fmul_rn(wk.one_m_alpha2, yy));
@@ -228,87 +276,147 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint64_t
     }
 }
 
-constexpr int kDecThreads = 128;
-#ifndef DQ_DEC_MINBLOCKS
-#define DQ_DEC_MINBLOCKS 4
-#endif
-constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;
-
+// ---------------------------------------------------------------------------------------------------
+// The decode kernel.  Grid = persistent CTAs of four autonomous warps; dynamic shared memory = kDecSmemBytes.
+// side_map / out_map: [whole rows x 32 floats] views of the caller's side information and output (valid when
+// args.use_tiles; side_map only when args.has_side).
+// ---------------------------------------------------------------------------------------------------
 template <int DITH, bool RUN>
 __global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
-decode_aggregate_kernel(const __grid_constant__ DecodeArgs args)
+decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __grid_constant__ CUtensorMap out_map,
+                        const __grid_constant__ DecodeArgs args)
 {
-    // Side information of the CTA's 128 rows -> shared memory (coalesced loads, 16-byte pieces swizzled so
-    // that "lane r reads row r" is free of bank conflicts); every worker then re-reads it from there.
-    __shared__ __align__(16) float side_tile[RUN ? 4 : kDecThreads * 32];
-    grid_dependency_wait();
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_side_mem[kDecWarps][kDecTileBuffers];
+
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t lane = threadIdx.x & 31u;
     grid_dependency_launch_next();
-    const uint64_t row0 = args.first_row + (uint64_t)blockIdx.x * blockDim.x;
-    {
-        // Ask the L2 for what the CTA that runs `prefetch_blocks` blocks later (one block per SM ahead) will load
-        // first: its side information and every message's words, so that those loads find their lines
-        // in the L2 instead of waiting for HBM.
-        const uint64_t frow0 = row0 + (uint64_t)args.prefetch_blocks * kDecThreads;
-        if (frow0 + threadIdx.x < args.rows) {
-            if (!RUN && args.side != nullptr) prefetch_l2(args.side + (frow0 + threadIdx.x) * 32u);
-        }
-        const uint32_t lane = threadIdx.x & 31u;
-        for (uint32_t w = threadIdx.x >> 5; w < args.W; w += (uint32_t)kDecThreads / 32u) {
-            const uint64_t first_word = frow0 * args.w[w].bits + 32u * lane;          // lines of 32 words
-            if (lane < 4u * args.w[w].bits && first_word < args.rows * args.w[w].bits)
-                prefetch_l2(args.w[w].packed + first_word);
-        }
-    }
-    if (!RUN && args.side != nullptr) {
-        // kDecThreads rows x 8 pieces = 8 pieces per thread
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t tiles = smem_base + warp * (uint32_t)(kDecTileBuffers * kDecTileBytes);
+    const uint32_t bar_side = smem_u32(&bar_side_mem[warp][0]);
+    const bool side_tiles = !RUN && args.has_side != 0u && args.use_tiles != 0u;
+
+    if (lane == 0) {
 #pragma unroll
-        for (uint32_t k = 0; k < 8u; ++k) {
-            const uint32_t q = threadIdx.x + (uint32_t)kDecThreads * k;       // 16-byte piece inside the CTA's block
-            const uint64_t piece = row0 * 8u + q;
-            if (piece * 4u + 4u <= args.n) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(args.side) + piece);
-                const uint32_t r = q >> 3, c = q & 7u;
-                *reinterpret_cast<float4*>(side_tile + r * 32u + ((c ^ (r & 7u)) << 2)) = v;
+        for (int i = 0; i < kDecTileBuffers; ++i) mbar_init(bar_side + 8u * i, 1u);
+        fence_mbar_init();
+        if (args.use_tiles) asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&out_map) : "memory");
+        if (side_tiles) asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&side_map) : "memory");
+    }
+    // the messages (and the side information) may be the previous kernel's output
+    grid_dependency_wait();
+
+    const uint32_t total_warps = gridDim.x * (uint32_t)kDecWarps;
+    const uint32_t gw = blockIdx.x * (uint32_t)kDecWarps + warp;
+    if (gw >= args.num_units) return;
+    const uint32_t my_units = (args.num_units - gw - 1u) / total_warps + 1u;
+    const uint32_t whole_rows = args.full_rows - args.first_row;       // rows of the tile maps
+
+    // side information of this warp's k-th unit -> tile buffer k mod 3 (lane 0)
+    auto issue_side = [&](uint32_t k) {
+        if ((gw + k * total_warps) * 32u >= whole_rows) return;         // a unit that is only the ragged last row
+        const uint32_t b = k % (uint32_t)kDecTileBuffers;
+        mbar_expect_tx(bar_side + 8u * b, (uint32_t)kDecTileBytes);
+        tma_load_rows(tiles + b * (uint32_t)kDecTileBytes, &side_map, bar_side + 8u * b,
+                      (int32_t)((gw + k * total_warps) * 32u));
+    };
+    // Ask the L2 for every worker's packed words of the unit that starts at row `row0`: lane w (and w + 32)
+    // requests the 128-byte lines of worker w, whose words of a unit are 128 * bits contiguous bytes.
+    auto prefetch_words = [&](uint32_t row0) {
+        if (row0 >= args.full_rows) return;
+        for (uint32_t w = lane; w < args.W; w += 32u) {
+            const uint32_t* p = args.w[w].packed + (uint64_t)row0 * args.w[w].bits;
+            const uint32_t rows_left = args.full_rows - row0;
+            const uint32_t lines = (rows_left >= 32u) ? args.w[w].bits : (rows_left * args.w[w].bits + 31u) / 32u;
+            for (uint32_t l = 0; l < lines; ++l) prefetch_l2(p + 32u * l);
+        }
+    };
+    if (lane == 0 && side_tiles) issue_side(0u);
+    __syncwarp();
+
+    // bucket of a row (rows past the end take the last row's bucket: their results are never stored)
+    auto bucket_of = [&](uint32_t r) {
+        const uint32_t rc = (r < args.rows) ? r : args.rows - 1u;
+        return (args.rpb_shift != 0xFFFFFFFFu) ? (rc >> args.rpb_shift) : (rc / args.rows_per_bucket);
+    };
+
+    const uint32_t swz16 = (lane & 7u) << 4;
+    bool gave_up = false;
+    uint32_t bucket = bucket_of(args.first_row + gw * 32u + lane);
+    float kappa_next = __ldg(args.w[0].scale + bucket);
+
+#pragma unroll 1
+    for (uint32_t k = 0; k < my_units; ++k) {
+        const uint32_t unit = gw + k * total_warps;
+        const uint32_t row = args.first_row + unit * 32u + lane;
+        const uint32_t b = k % (uint32_t)kDecTileBuffers;
+        const uint32_t tile = tiles + b * (uint32_t)kDecTileBytes;
+        const bool more = k + 1u < my_units;
+        const uint32_t bucket_next = more ? bucket_of(row + total_warps * 32u) : bucket;
+        if (more) prefetch_words(row - lane + total_warps * 32u);
+        if (lane == 0) {
+            // the store issued two units ago has read its buffer: that buffer takes the next unit's side
+            // information now and this unit's output later
+            bulk_wait_group_read<1>();
+            if (side_tiles && more) issue_side(k + 1u);
+        }
+        __syncwarp();
+        const bool unit_has_tile = unit * 32u < whole_rows;
+        if (side_tiles && unit_has_tile &&
+            !mbar_wait_bounded(bar_side + 8u * b, (k / (uint32_t)kDecTileBuffers) & 1u, gave_up)) {
+            gave_up = true;
+            if (lane == 0) atomicOr(args.error_flags, 0x2u);
+        }
+        const uint32_t row_addr = (tile + lane * 128u) | swz16;
+        // lanes past the last whole row compute on the last whole row's words (in bounds) and are never stored
+        const uint32_t load_row = (row < args.full_rows) ? row : args.full_rows - 1u;
+
+        float acc[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
+        uint32_t kappa_bits_max = 0u;
+
+        if (unit_has_tile) {
+#pragma unroll 1
+            for (uint32_t w = 0; w < args.W; ++w) {
+                const float kappa = kappa_next;
+                // the next step's scale: the next worker's for this bucket, or the first worker's for the next unit
+                kappa_next = (w + 1u < args.W) ? __ldg(args.w[w + 1u].scale + bucket)
+                                               : __ldg(args.w[0].scale + bucket_next);
+                decode_row_variant<DITH, RUN>(args.w[w], row, load_row, kappa, row_addr, acc, args.half_bias_bits);
+                const uint32_t kb = __float_as_uint(kappa) & 0x7FFFFFFFu;
+                kappa_bits_max = (kb > kappa_bits_max) ? kb : kappa_bits_max;
             }
+        } else {
+            kappa_next = __ldg(args.w[0].scale + bucket_next);
         }
-        __syncthreads();
-    }
+        bucket = bucket_next;
 
-    const uint64_t row = row0 + threadIdx.x;
-    if (row >= args.rows) return;
-    const uint64_t base = row * 32u;
-    const uint64_t bucket = row / args.rows_per_bucket;
-    if (base + 32u > args.n) {
-        decode_partial_row<DITH, RUN>(args, row, bucket, (uint32_t)(args.n - base));
-        return;
-    }
-    const float* side_row = side_tile + (RUN ? 0u : threadIdx.x * 32u);
-
-    float acc[32];
+        // the mean leaves through the tile buffer: the lane writes its row where it read its side information
 #pragma unroll
-    for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
-
-    for (uint32_t w = 0; w < args.W; ++w) {
-        const DecWorker& wk = args.w[w];
-        uint32_t cur[8];
-        float kappa;
-        load_worker_row(wk, row, bucket, cur, kappa);
-        switch (wk.kind) {
-            case kDecDqsg: decode_row_bits<kDecDqsg, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
-            case kDecNdqsgPow2: decode_row_bits<kDecNdqsgPow2, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
-            case kDecNdqsgPow2Shrink: decode_row_bits<kDecNdqsgPow2Shrink, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
-            default: decode_row_bits<kDecNdqsgAnyK, DITH, RUN>(wk, row, cur, kappa, side_row, acc, args.status, args.half_bias_bits); break;
+        for (int c = 0; c < 8; ++c) {
+            float v[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                v[e] = (args.invW != 0.0f) ? __fmul_rn(acc[4 * c + e], args.invW) : __fdiv_rn(acc[4 * c + e], args.Wf);
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
+                         ::"r"(row_addr ^ (uint32_t)(c << 4)), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3])
+                         : "memory");
         }
+        fence_proxy_async_shared();
+        __syncwarp();
+        if (lane == 0 && unit_has_tile) {
+            tma_store_rows(&out_map, tile, (int32_t)(unit * 32u));
+            bulk_commit_group();
+        }
+        if (args.status != nullptr && kappa_bits_max >= 0x7F800000u && row < args.full_rows) atomicOr(args.status, 0x1u);
+        if (row == args.full_rows && row < args.rows)
+            decode_partial_row<DITH, RUN>(args, row, bucket_of(row), (uint32_t)(args.n - (uint64_t)row * 32u));
     }
-
-#pragma unroll
-    for (int e = 0; e < 32; ++e)
-        acc[e] = (args.invW != 0.0f) ? __fmul_rn(acc[e], args.invW) : __fdiv_rn(acc[e], args.Wf);
-
-#pragma unroll
-    for (int c = 0; c < 8; ++c)
-        reinterpret_cast<float4*>(args.out + base)[c] =
-            make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+    // shared memory must stay valid until the last stores have read it
+    if (lane == 0) bulk_wait_group_read<0>();
 }
 
 }  // namespace dq

@@ -228,25 +228,79 @@ __device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap* t
         : "memory");
 }
 
-// Upper bound, in nanoseconds, that one try may stay suspended in hardware before it reports "not yet".
-constexpr uint32_t kWaitHintNs = 20000u;
-
-// Waits for phase `parity` of the barrier; gives up after a fixed number of tries (each try itself blocks
-// for a hardware-defined time), so a copy that never lands cannot hang the kernel.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t max_tries = (1u << 22))
+// Contiguous bulk copy global -> shared memory (both addresses 16-byte aligned, size a multiple of 16 bytes).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
-    for (uint32_t it = 0; it < max_tries; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity), "r"(kWaitHintNs)
-            : "memory");
-        if (ok) return true;
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Store a [32 rows x 32 floats] box from shared memory (128-byte swizzle) to rows row0.. of the mapped array; rows
+// past the array's end are not written.  Completion is tracked by the issuing thread's bulk groups.
+__device__ __forceinline__ void tma_store_rows(const CUtensorMap* tmap, uint32_t src, int32_t row0)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"((uint64_t)tmap), "r"(src), "r"(0), "r"(row0)
+                 : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit_group()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+// Waits until at most N of this thread's bulk groups still have to read their shared-memory source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+// Makes this thread's earlier shared-memory writes visible to the asynchronous copy engine.
+__device__ __forceinline__ void fence_proxy_async_shared()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Upper bound, in nanoseconds, that one try may stay suspended in hardware before it reports "not yet".
+constexpr uint32_t kWaitHintNs = 2000u;
+// A copy that has not landed after this long (by the global nanosecond timer) is given up: a tile copy takes
+// microseconds, so 20 ms means that it will never arrive.
+constexpr uint64_t kWaitGiveUpNs = 20ull * 1000ull * 1000ull;
+
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(kWaitHintNs)
+        : "memory");
+    return ok != 0u;
+}
+
+// Waits for phase `parity` of the barrier, but not for ever: after kWaitGiveUpNs (or after a single try when
+// `single_try` is set, which callers do once a wait has already run out) it returns false, so a copy that never
+// lands cannot hang the kernel.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, bool single_try = false)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    if (single_try) return false;
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - t0 > kWaitGiveUpNs) return false;
     }
-    return false;
 }
 
 // Named barrier over `threads` threads (a multiple of 32); id 1..15 (0 is __syncthreads).
@@ -258,13 +312,6 @@ __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
 __device__ __forceinline__ void prefetch_l2(const void* p)
 {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
-
-__device__ __forceinline__ uint64_t global_timer_ns()
-{
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
 }
 
 // Programmatic dependent launch: wait until the previous kernel of the stream has completed and its writes are

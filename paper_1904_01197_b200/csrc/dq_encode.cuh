@@ -436,8 +436,8 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
             for (uint32_t half = 0; half < 2u; ++half) {
                 const uint32_t stage_addr = (my_smem + half * kWarpTileBytes + lane * 128u) | swz16;
                 if (half == 0u) {
-                    if (!mbar_wait_bounded(my_bar, par, gave_up ? 1u : (1u << 22)) ||
-                        !mbar_wait_bounded(my_bar + 8u, par, gave_up ? 1u : (1u << 22))) {
+                    if (!mbar_wait_bounded(my_bar, par, gave_up) ||
+                        !mbar_wait_bounded(my_bar + 8u, par, gave_up)) {
                         gave_up = true;
                         if (lane == 0) atomicOr(args.error_flags, 0x2u);
                     }
@@ -506,7 +506,7 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
     for (uint64_t tile = first_tile; tile < args.num_units; tile += stride, ++k) {
         const uint32_t s = k % kEncStages;
         const uint32_t use = k / kEncStages;
-        if (!mbar_wait_bounded(my_bar + 8u * s, use & 1u, gave_up ? 1u : (1u << 22))) {
+        if (!mbar_wait_bounded(my_bar + 8u * s, use & 1u, gave_up)) {
             gave_up = true;
             if (lane == 0) atomicOr(args.error_flags, 0x2u);
         }

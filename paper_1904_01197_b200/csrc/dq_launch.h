@@ -45,8 +45,10 @@ DQ_DECLARE_ENCODE(0, 16) DQ_DECLARE_ENCODE(1, 16) DQ_DECLARE_ENCODE(2, 16) DQ_DE
 #undef DQ_DECLARE_ENCODE
 
 // Decoder: dith = 32, 16 or 0 (no dither at the receiver); run = side information is the running mean.
+// The grid (persistent CTAs) follows from a.num_units and the device.
 #define DQ_DECLARE_DECODE(DITH, RUN)                                                                               \
-    cudaError_t launch_decode_d##DITH##_r##RUN(const DecodeArgs& a, uint32_t grid, cudaStream_t st);
+    cudaError_t launch_decode_d##DITH##_r##RUN(const CUtensorMap& side_map, const CUtensorMap& out_map,            \
+                                               const DecodeArgs& a, int sm_count, cudaStream_t st);
 DQ_DECLARE_DECODE(32, 0) DQ_DECLARE_DECODE(32, 1) DQ_DECLARE_DECODE(16, 0) DQ_DECLARE_DECODE(16, 1)
 DQ_DECLARE_DECODE(0, 0)
 #undef DQ_DECLARE_DECODE
