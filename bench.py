@@ -35,24 +35,31 @@ if str(ROOT) not in sys.path:
 METRIC = "encode / fused decode-aggregate GB/s and % of HBM peak on 1 B200; Gelem/s"
 L2_BYTES = 126 * 1024 * 1024
 HBM_NOMINAL_GBS = 8000.0
-SM_COUNT, ISSUE_PER_SM_CLK, LANES = 148, 4, 32           # ALU-issue ceiling: SMs x schedulers x lanes x clock
-# Algorithmic lane-instructions: ~22 per (element, worker) + ~10 per element for the fused decode,
-# ~24 per element for the encode.
+SM_COUNT, ISSUE_PER_SM_CLK, LANES = 148, 4, 32           # issue ceiling: SMs x schedulers x lanes x clock
+# Algorithmic lane-instructions of the method itself: a quarter of a Philox block per dither value (4.5 wide
+# multiplies + 4.75 three-input XORs), the dither conversion (2), and for the fused decode unpacking (3) plus 5
+# (DQSG) to 9 (NDQSG) fp32 operations per (element, worker), about 10 per element for the mean and the stores;
+# for the encode 24 per element with the scale reduction and the packing.
 DEC_INSTR_PER_ELEM_WORKER, DEC_INSTR_PER_ELEM, ENC_INSTR_PER_ELEM = 22.0, 10.0, 24.0
-# Executed lane-instructions per (element, worker) of the fused decode on the ResNet-50-sized workload, from the
-# opcode counters in profiles/decode_aggregate_kernel_ndqsg_resnet50.md: (32x32->64 multiplies, fp32 adds /
-# multiplies / multiply-adds, everything else).  Their scheduler cost is taken from the issue probe
-# (profiles/issue_cost_probe_b200.md): 4.4 cycles per wide multiply with one other instruction hidden behind it,
-# 1 cycle per fp32 instruction, 2 cycles for the rest; the classes add up.
-DEC_MIX = {32: (4.34, 9.82, 12.52), 16: (2.20, 9.82, 9.88)}
-ISSUE_CYCLES_WIDE, ISSUE_CYCLES_FP32, ISSUE_CYCLES_OTHER = 4.4, 1.0, 2.0
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
-# profiles/; keyed by (kernel class, workload, n).  None once a kernel has changed since its capture.
-NCU_TRAFFIC = {
-    ("encode", "ndqsg_resnet50", 25_557_032, 2): 106_543_616,    # profiles/encode_kernel_ndqsg_resnet50.md
-    ("encode", "ndqsg_resnet50", 25_557_032, 3): 106_651_648,
-    ("decode", "ndqsg_resnet50", 25_557_032): 223_945_472,       # profiles/decode_aggregate_kernel_ndqsg_resnet50.md
-}
+FLAG_INPUT_READY, FLAG_OUTPUT_FREE = 1, 2
+
+
+def source_hash():
+    from paper_1904_01197_b200 import build as dq_build
+    return dq_build.source_hash()
+
+
+def committed_counters():
+    """Counters taken from committed profiler summaries (profiles/counters_*.md): lines of the form
+    `counter: <name> <value> csrc=<hash>`.  A counter is returned only if the library's sources still have the
+    content hash it was captured at; otherwise the kernel has changed and the value is unknown (None)."""
+    out, now = {}, source_hash()
+    for f in sorted((ROOT / "profiles").glob("counters_*.md")):
+        for line in f.read_text().splitlines():
+            parts = line.strip().split()
+            if len(parts) >= 4 and parts[0] == "counter:" and parts[3].startswith("csrc="):
+                out[parts[1]] = float(parts[2]) if parts[3] == f"csrc={now}" else None
+    return out
 
 
 def parse_args():
@@ -70,6 +77,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-kernels", action="store_true", help="skip the per-kernel isolated timings")
+    ap.add_argument("--no-other", action="store_true", help="skip the compact record of the other workloads")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under a profiler: only warm-up + timed steps, no sampler, no extra legs")
     ap.add_argument("--cpu-sample", type=int, default=1 << 25, help="elements per worker in the oracle sample")
@@ -183,9 +191,15 @@ class GpuState:
         from dq_workloads.generators import DQSG
         self.dq, self.torch, self.cfg, self.dev = dq, torch, cfg, dev
         self.DQSG = DQSG
-        self.params = [dq.binding.make_params(cfg.bucket, s.bits, s.levels, s.coarse_K, s.fine_M, s.alpha,
-                                              s.dither_bits)
-                       for s in cfg.workers]
+        mk = lambda s, flags=0: dq.binding.make_params(cfg.bucket, s.bits, s.levels, s.coarse_K, s.fine_M, s.alpha,
+                                                       s.dither_bits, flags)
+        self.params = [mk(s) for s in cfg.workers]
+        # Inside a step the gradients are complete long before the encodes start, and the encode of worker w
+        # writes buffers that the encode of worker w - 1 does not touch: every encode may read early, and all but
+        # the first (whose message buffer the previous step's decode may still be reading) may also store early.
+        self.step_params = [mk(s, FLAG_INPUT_READY | (FLAG_OUTPUT_FREE if w > 0 else 0))
+                            for w, s in enumerate(cfg.workers)]
+        self.overlap_params = [mk(s, FLAG_INPUT_READY | FLAG_OUTPUT_FREE) for s in cfg.workers]
         if share is not None:
             self.grads_host, self.grads = share.grads_host, share.grads
         else:
@@ -209,8 +223,8 @@ class GpuState:
         self.out = torch.empty(cfg.n, dtype=torch.float32, device=dev)
         torch.cuda.synchronize()
 
-    def encode(self, w, grad=None, bufs=None):
-        s, p = self.cfg.workers[w], self.params[w]
+    def encode(self, w, grad=None, bufs=None, params=None):
+        s, p = self.cfg.workers[w], (self.params[w] if params is None else params)
         pk, sc = bufs if bufs is not None else self.msg_buf[w]
         fn = self.dq.dqsg_encode if s.kind == self.DQSG else self.dq.ndqsg_encode
         fn(self.grads[w] if grad is None else grad, s.seed, w, self.cfg.step, p, pk, sc)
@@ -226,18 +240,30 @@ class GpuState:
         else:
             self.dq.dqsg_decode_aggregate(msgs, self.cfg.n, self.cfg.step, out)
 
-    def step(self, ev_mid=None):
+    def decode_side_first(self, msgs=None, out=None):
+        self.dq.ndqsg_decode_aggregate_side_first(self.msgs if msgs is None else msgs, self.cfg.n, self.cfg.step,
+                                                  self.out if out is None else out)
+
+    def step(self, ev_mid=None, two_call=False, plain_launches=False):
+        """One pass of the whole path.  When the side information is worker 0's reconstruction it is taken
+        inside the fused decode (one launch); two_call=True runs the W=1 decode and the fused decode with a side
+        information vector instead.  plain_launches=True encodes without the early-read / early-store flags."""
         for w in range(self.cfg.W):
-            self.encode(w)
+            self.encode(w, params=None if plain_launches else self.step_params[w])
         if ev_mid is not None:
             ev_mid.record()
-        if self.cfg.side_from_worker0:
-            self.side_decode()
-        self.decode()
+        if self.cfg.side_from_worker0 and not two_call:
+            self.decode_side_first()
+        else:
+            if self.cfg.side_from_worker0:
+                self.side_decode()
+            self.decode()
 
-    def step_bytes(self):
+    def step_bytes(self, two_call=False):
         cfg, dq = self.cfg, self.dq
         enc = sum(encode_bytes(dq, cfg.n, s, cfg.bucket) for s in cfg.workers)
+        if cfg.side_from_worker0 and not two_call:
+            return enc, decode_bytes(dq, cfg.n, cfg.workers, cfg.bucket, False)
         dec = decode_bytes(dq, cfg.n, cfg.workers, cfg.bucket, self.any_nested)
         if cfg.side_from_worker0:
             dec += decode_bytes(dq, cfg.n, cfg.workers[:1], cfg.bucket, False)
@@ -269,18 +295,27 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
     for w, s in enumerate(cfg.workers):
         key = (s.kind, s.bits, s.levels, s.coarse_K)
         seen.setdefault(key, w)
-    rot = max(1, min(cfg.W, -(-3 * L2_BYTES // (4 * n))))
+    rot = max(2, min(cfg.W, -(-3 * L2_BYTES // (4 * n))))
+    counters = committed_counters()
     for key, w in seen.items():
         s = cfg.workers[w]
-        launches = [(lambda gg=st.grads[(w + r) % cfg.W], ww=w: st.encode(ww, grad=gg)) for r in range(rot)]
-        ms = time_isolated(torch, launches)
         by = encode_bytes(dq, n, s, cfg.bucket)
         name = f"encode_{'dqsg' if s.kind == st.DQSG else 'ndqsg'}_b{s.bits}"
-        res[name] = {"ms": ms, "bytes": by, "gbs": by / ms / 1e6, "gelem_s": n / ms / 1e6,
-                     "frac_hbm": by / ms / 1e6 / hbm_peak, "rotating_buffers": rot,
-                     "alu_tinstr_s": ENC_INSTR_PER_ELEM * n / ms / 1e9,
-                     "frac_alu": ENC_INSTR_PER_ELEM * n / ms * 1e3 / alu_peak,
-                     "traffic": NCU_TRAFFIC.get(("encode", cfg.name, n, s.bits)) if s.dither_bits == 32 else None}
+        # rotating inputs AND outputs: consecutive launches share nothing, as the overlapped variant requires
+        outs = [dq.binding.alloc_message(n, st.params[w], st.dev) for _ in range(rot)]
+        for variant, params in (("", st.params[w]), ("_overlapped", st.overlap_params[w])):
+            launches = [(lambda gg=st.grads[(w + r) % cfg.W], ww=w, oo=outs[r], pp=params:
+                         st.encode(ww, grad=gg, bufs=oo, params=pp)) for r in range(rot)]
+            ms = time_isolated(torch, launches)
+            res[name + variant] = {
+                "ms": ms, "bytes": by, "gbs": by / ms / 1e6, "gelem_s": n / ms / 1e6,
+                "frac_hbm": by / ms / 1e6 / hbm_peak, "rotating_buffers": rot,
+                "launch_flags": ("DQ_FLAG_INPUT_READY|DQ_FLAG_OUTPUT_FREE: back-to-back launches overlap"
+                                 if variant else "none: each launch waits for the previous one"),
+                "alu_tinstr_s": ENC_INSTR_PER_ELEM * n / ms / 1e9,
+                "frac_alu": ENC_INSTR_PER_ELEM * n / ms * 1e3 / alu_peak,
+                "traffic": counters.get(f"{cfg.name}.{name}.dram_bytes") if s.dither_bits == 32 else None}
+        del outs
     # decode: rotate over message sets / side / out copies so that nothing is L2-resident
     per_set = decode_bytes(dq, n, cfg.workers, cfg.bucket, st.any_nested)
     sets = max(2, min(6, -(-3 * L2_BYTES // per_set)))
@@ -296,6 +331,24 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
         outs.append(torch.empty_like(st.out))
     launches = [(lambda a=msg_sets[i], b=sides[i], c=outs[i]: st.decode(a, b, c)) for i in range(sets)]
     ms = time_isolated(torch, launches, iters=12)
+
+    def entry(ms_, by_, workers):
+        return {"ms": ms_, "bytes": by_, "gbs": by_ / ms_ / 1e6, "gelem_s": n / ms_ / 1e6,
+                "frac_hbm": by_ / ms_ / 1e6 / hbm_peak, "gelem_worker_s": n * workers / ms_ / 1e6}
+
+    if cfg.side_from_worker0:
+        # the side information taken from message 0 inside the fused pass (no vector read, no W = 1 launch)
+        sf_l = [(lambda a=msg_sets[i], c=outs[i]: st.decode_side_first(a, c)) for i in range(sets)]
+        res["decode_aggregate_side_first"] = entry(time_isolated(torch, sf_l, iters=12), per_set - 4 * n, cfg.W)
+    # the first message alone (W = 1): the P1 decode of Algorithm 2, and the small-W end of the decoder
+    by_w1 = decode_bytes(dq, n, cfg.workers[:1], cfg.bucket, cfg.workers[0].kind != st.DQSG)
+    w1_sets = max(2, min(8, -(-3 * L2_BYTES // by_w1)))
+    w1_outs = [torch.empty_like(st.out) for _ in range(max(0, w1_sets - sets))] + outs
+    w1_l = [(lambda a=msg_sets[i % sets][:1], b=sides[i % sets], c=w1_outs[i]:
+             (dq.ndqsg_decode_aggregate(a, n, cfg.step, b, c) if cfg.workers[0].kind != st.DQSG
+              else dq.dqsg_decode_aggregate(a, n, cfg.step, c))) for i in range(w1_sets)]
+    res["decode_aggregate_w1"] = entry(time_isolated(torch, w1_l, iters=16), by_w1, 1)
+    del w1_outs
     if not st.any_nested:
         # the receiver without the dither (no random numbers): the memory-bound limit of the decoder
         half_l = [(lambda a=msg_sets[i], c=outs[i]: dq.dqsg_decode_aggregate_half_dithered(a, n, c)) for i in range(sets)]
@@ -332,9 +385,48 @@ def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):
                                "gelem_worker_s": elem_workers / ms / 1e6, "rotating_buffers": sets,
                                "alu_tinstr_s": alg_instr / ms / 1e9, "frac_alu": alg_instr / ms * 1e3 / alu_peak,
                                "alu_peak_tinstr_s": alu_peak / 1e12,
-                               "traffic": (NCU_TRAFFIC.get(("decode", cfg.name, n))
+                               "traffic": (counters.get(f"{cfg.name}.decode_aggregate.dram_bytes")
                                            if cfg.workers[0].dither_bits == 32 else None)}
     return res
+
+
+def other_workloads(torch, hbm_peak, sm_max_mhz):
+    """Compact record of the other workload shapes: the ResNet-18-sized DQSG and the GPT-2-small-sized NDQSG
+    configurations, three points of the bandwidth sweep (n = 2^26; W = 2, 8, 32), and the issue probe's
+    Philox-only and kernel-mix ceilings.  Gradients are N(0,1) drawn on the device (timing only)."""
+    from bench_tools import sweep
+    keep = ("encode_us", "encode_gbs", "encode_frac_hbm", "decode_us", "decode_gbs", "decode_frac_hbm",
+            "decode_gelem_worker_s")
+    pts = {"dqsg_resnet18_b2": dict(n=11_689_512, W=8, bits=2, bucket=2048, kind="dqsg"),
+           "ndqsg_gpt2_small": dict(n=124_439_808, W=16, bits=3, bucket=4096, kind="ndqsg"),
+           "sweep_n2^26_W2": dict(n=1 << 26, W=2, bits=2, bucket=2048, kind="ndqsg"),
+           "sweep_n2^26_W8": dict(n=1 << 26, W=8, bits=2, bucket=2048, kind="ndqsg"),
+           "sweep_n2^26_W32": dict(n=1 << 26, W=32, bits=2, bucket=2048, kind="ndqsg")}
+    out = {}
+    for name, pt in pts.items():
+        try:
+            r = sweep.run_point(dither_bits=32, hbm_peak=hbm_peak, iters=8, **pt)
+            out[name] = dict(pt, **{k: r[k] for k in keep})
+        except Exception as e:                       # an out-of-memory point must not lose the line
+            out[name] = dict(pt, error=str(e)[:200])
+        torch.cuda.empty_cache()
+    try:
+        from bench_tools import issue_probe
+        exe = issue_probe.build()
+        probe = {}
+        for key in ("wide", "round", "dec_coarse", "enc_coarse"):
+            txt = subprocess.run([str(exe), key, "4"], capture_output=True, text=True, timeout=120).stdout
+            probe[key + "_cycles"] = float(txt.split("instr")[1].split("cycles/group")[0])
+        sched_hz = SM_COUNT * ISSUE_PER_SM_CLK * sm_max_mhz * 1e6
+        out["issue_probe"] = dict(
+            probe, what=("scheduler cycles per group, 4 warps per scheduler: one 32x32->64 multiply; one Philox "
+                         "round; the decoder's / encoder's instruction mix for 16 elements with nothing else"),
+            philox_only_gblocks_s=sched_hz * LANES / (9.0 * probe["round_cycles"]) / 1e9,
+            decode_mix_ceiling_gelem_worker_s=sched_hz * LANES * 16.0 / probe["dec_coarse_cycles"] / 1e9,
+            encode_mix_ceiling_gelem_s=sched_hz * LANES * 16.0 / probe["enc_coarse_cycles"] / 1e9)
+    except Exception as e:
+        out["issue_probe"] = {"error": str(e)[:200]}
+    return out
 
 
 def run_e2e(st: GpuState, steps: int):
@@ -565,39 +657,73 @@ def main():
     if not args.no_e2e:
         dt, h2d, d2h, _ = run_e2e(st, max(1, min(args.steps, 3)))
         dt = max_over_ranks([dt], dev)[0]
-        e2e = {"value": world * step_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+        e2e_bytes = sum(st.step_bytes(two_call=True))          # the host path decodes message 0 in a call of its own
+        e2e = {"value": world * e2e_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3}
+
+    # the step as two decode calls (W = 1 pass writes the side information, the fused pass reads it) and with
+    # plain launches: the form without the fused side information and without the launch flags
+    variants = None
+    if not args.profile and cfg.side_from_worker0:
+        for _ in range(3):
+            st.step(two_call=True, plain_launches=True)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            st.step(two_call=True, plain_launches=True)
+        e1.record()
+        torch.cuda.synchronize()
+        ms2 = max_over_ranks([e0.elapsed_time(e1) / args.steps], dev)[0]
+        by2 = sum(st.step_bytes(two_call=True))
+        variants = {"two_decode_calls_plain_launches": {"ms_per_step": ms2, "bytes": by2,
+                                                        "value": whole_job_value(by2, world, ms2), "unit": "GB/s",
+                                                        "launches_per_step": cfg.W + 2}}
+    other = None
+    if rank == 0 and not args.no_kernels and not args.no_other and args.workload == "ndqsg_resnet50":
+        del st.msg_buf, st.msgs
+        torch.cuda.empty_cache()
+        other = other_workloads(torch, hbm_peak, sm_max_mhz)
 
     if rank == 0:
         n_enc = cfg.W
         enc_share = enc_ms / (enc_ms + dec_ms)
         roofline_encode = None
         if kernels:
-            # the dominant kernel = the one with the largest share of the step's device time
-            enc_names = [k for k in kernels if k.startswith("encode")]
+            enc_names = [k for k in kernels if k.startswith("encode") and not k.endswith("_overlapped")]
             count = {k: sum(1 for s in cfg.workers if k == f"encode_{'dqsg' if s.kind == 0 else 'ndqsg'}_b{s.bits}")
                      for k in enc_names}
             dom_enc = max(enc_names, key=lambda k: count[k] * kernels[k]["ms"])
-            ke, kd = kernels[dom_enc], kernels["decode_aggregate"]
+            # encode: the launch as the step issues it (inputs ready, outputs free: launches overlap)
+            ke, ke_plain = kernels[dom_enc + "_overlapped"], kernels[dom_enc]
+            dec_name = "decode_aggregate_side_first" if cfg.side_from_worker0 else "decode_aggregate"
+            kd = kernels[dec_name]
             roofline_encode = {"kernel": dom_enc, "bound": "hbm", "achieved": ke["gbs"], "peak": hbm_peak,
                                "unit": "GB/s", "frac": ke["gbs"] / hbm_peak, "traffic": ke["traffic"],
                                "peak_source": f"of {peak_src}", "frac_of_nominal_8TBs": ke["gbs"] / HBM_NOMINAL_GBS,
-                               "launches_per_step": count[dom_enc], "frac_alu": ke["frac_alu"]}
-            roofline_decode = {"kernel": "decode_aggregate", "bound": "alu", "achieved": kd["alu_tinstr_s"],
-                               "peak": kd["alu_peak_tinstr_s"], "unit": "Tlane-instr/s", "frac": kd["frac_alu"],
-                               "traffic": kd["traffic"],
+                               "launches_per_step": count[dom_enc], "launch_flags": ke["launch_flags"],
+                               "us_per_launch": ke["ms"] * 1e3,
+                               "without_flags": {"achieved": ke_plain["gbs"], "frac": ke_plain["frac_hbm"],
+                                                 "us_per_launch": ke_plain["ms"] * 1e3}}
+            # decode: bound by instruction issue; algorithmic lane-instructions against the issue ceiling, and the
+            # multiplier pipe beside it (a 32x32->64 multiply holds it for four cycles, 4.5 of them per dither value)
+            alu_peak = SM_COUNT * ISSUE_PER_SM_CLK * LANES * sm_max_mhz * 1e6
+            alg_instr = DEC_INSTR_PER_ELEM_WORKER * cfg.n * cfg.W + DEC_INSTR_PER_ELEM * cfg.n
+            cyc_per_unit = SM_COUNT * ISSUE_PER_SM_CLK * LANES * sm_max_mhz * 1e6 / (kd["gelem_worker_s"] * 1e9)
+            dith = cfg.workers[0].dither_bits
+            wide_per_unit = 18.0 / (4 if dith == 32 else 8)
+            roofline_decode = {"kernel": dec_name, "bound": "alu", "achieved": alg_instr / kd["ms"] / 1e9,
+                               "peak": alu_peak / 1e12, "unit": "Tlane-instr/s",
+                               "frac": alg_instr / kd["ms"] * 1e3 / alu_peak,
+                               "traffic": kernels["decode_aggregate"].get("traffic") if dec_name == "decode_aggregate" else None,
                                "peak_source": "148 SMs x 4 schedulers x 32 lanes x max SM clock",
-                               "hbm_gbs": kd["gbs"], "frac_hbm": kd["frac_hbm"], "launches_per_step": 1}
-            mix = DEC_MIX.get(cfg.workers[0].dither_bits)
-            if mix and cfg.name == "ndqsg_resnet50":
-                wide, fp32, other = mix
-                cycles = (ISSUE_CYCLES_WIDE * wide + ISSUE_CYCLES_FP32 * fp32 +
-                          ISSUE_CYCLES_OTHER * max(0.0, other - wide))
-                ceiling = SM_COUNT * ISSUE_PER_SM_CLK * LANES * sm_max_mhz * 1e6 / cycles
-                roofline_decode["issue_mix"] = {"wide_mul_per_unit": wide, "fp32_instr_per_unit": fp32,
-                                                "other_instr_per_unit": other, "scheduler_cycles_per_unit": cycles,
-                                                "ceiling_gelem_worker_s": ceiling / 1e9,
-                                                "frac_of_ceiling": kd["gelem_worker_s"] * 1e9 / ceiling}
+                               "hbm_gbs": kd["gbs"], "frac_hbm": kd["frac_hbm"], "launches_per_step": 1,
+                               "gelem_worker_s": kd["gelem_worker_s"],
+                               "scheduler_cycles_per_element_worker": cyc_per_unit,
+                               "multiplier_pipe": {"wide_multiplies_per_element_worker": wide_per_unit,
+                                                   "pipe_cycles_per_wide_multiply": 4.0,
+                                                   "floor_cycles_per_element_worker": 4.0 * wide_per_unit,
+                                                   "frac": 4.0 * wide_per_unit / cyc_per_unit}}
             if kd["ms"] >= count[dom_enc] * ke["ms"]:
                 roofline = roofline_decode
             else:
@@ -623,6 +749,10 @@ def main():
             line["roofline_encode"] = roofline_encode
         if roofline_decode is not None and roofline_decode is not roofline:
             line["roofline_decode"] = roofline_decode
+        if variants is not None:
+            line["step_variants"] = variants
+        if other is not None:
+            line["other_workloads"] = other
         if alt is not None:
             line["dither16"] = alt
         if e2e:

@@ -154,6 +154,17 @@ dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uin
                                  void* cuda_stream);
 
 /*
+ * ndqsg_decode_aggregate_side_first -- the server of Algorithm 2 with one worker in P1: message 0 (which must be
+ * a DQSG message) is decoded first and its reconstruction g~_0 is the side information y of every NDQSG message
+ * that follows; the mean of all W reconstructions is written.  The result is bit-identical to
+ *     dqsg_decode_aggregate(msgs, 1, ..., y);  ndqsg_decode_aggregate(msgs, W, ..., y, out_avg, ...)
+ * but y never exists in global memory: no side-information vector is read and the first pass is not launched.
+ * Other arguments as for ndqsg_decode_aggregate.
+ */
+dq_status ndqsg_decode_aggregate_side_first(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                            float* out_avg, uint32_t* status_word, void* cuda_stream);
+
+/*
  * dqsg_decode_aggregate_half_dithered -- the receiver that cannot reproduce the dither (Section 2.1,
  * "half-dithered quantization" x~_h = Q(x + u); by Lemma 1 this is M-level stochastic quantization): every
  * DQSG message is reconstructed as kappa * Delta * q with nothing subtracted, and the mean is written.  No

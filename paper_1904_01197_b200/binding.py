@@ -69,6 +69,8 @@ def lib() -> C.CDLL:
         L.dqsg_decode_aggregate_half_dithered.restype = C.c_int
         L.ndqsg_decode_aggregate_running.argtypes = [pm, u32, u64, u64, vp, vp, vp]
         L.ndqsg_decode_aggregate_running.restype = C.c_int
+        L.ndqsg_decode_aggregate_side_first.argtypes = [pm, u32, u64, u64, vp, vp, vp]
+        L.ndqsg_decode_aggregate_side_first.restype = C.c_int
         L.dq_code_histogram.argtypes = [vp, u64, u32, vp, vp]
         L.dq_code_histogram.restype = C.c_int
         for f in (L.dqsg_encode_range, L.ndqsg_encode_range):
@@ -301,6 +303,19 @@ def ndqsg_decode_aggregate_running(msgs: Sequence[Message], n: int, step: int,
                                                 _dev_ptr(out_avg, torch.float32, "out_avg"),
                                                 _dev_ptr(status_word, torch.int32, "status_word"),
                                                 _stream_ptr(stream)), "ndqsg_decode_aggregate_running")
+    return out_avg
+
+
+def ndqsg_decode_aggregate_side_first(msgs: Sequence[Message], n: int, step: int,
+                                      out_avg: Optional[torch.Tensor] = None,
+                                      status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Algorithm 2 with one P1 worker: the reconstruction of message 0 is the side information of the rest."""
+    if out_avg is None:
+        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+    _check(lib().ndqsg_decode_aggregate_side_first(_msg_array(msgs), len(msgs), n, step,
+                                                   _dev_ptr(out_avg, torch.float32, "out_avg"),
+                                                   _dev_ptr(status_word, torch.int32, "status_word"),
+                                                   _stream_ptr(stream)), "ndqsg_decode_aggregate_side_first")
     return out_avg
 
 

@@ -32,7 +32,7 @@ UNITS = [("dq_b200", "dq_b200.cu", [])]
 UNITS += [(f"enc_m{m}_d{d}", "dq_encode_inst.cu", [f"-DDQ_INST_MODE={m}", f"-DDQ_INST_DITH={d}"])
           for m in (0, 1, 2, 3) for d in (32, 16)]
 UNITS += [(f"dec_d{d}_r{r}", "dq_decode_inst.cu", [f"-DDQ_INST_DITH={d}", f"-DDQ_INST_RUN={r}"])
-          for d, r in ((32, 0), (32, 1), (16, 0), (16, 1), (0, 0))]
+          for d, r in ((32, 0), (32, 1), (32, 2), (16, 0), (16, 1), (16, 2), (0, 0))]
 
 
 def nvcc_path() -> str:

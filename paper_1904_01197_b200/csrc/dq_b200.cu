@@ -277,7 +277,8 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
 
 dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, const float* side_info,
                         float* out_avg, uint32_t* status_word, bool allow_nested, cudaStream_t st,
-                        bool running = false, bool half_dithered = false, uint64_t first_element = 0u)
+                        bool running = false, bool half_dithered = false, uint64_t first_element = 0u,
+                        bool side_first = false)
 {
     if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
     static thread_local dq::DecodeArgs a;    // ~10 KB: keep it off the stack
@@ -330,13 +331,15 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     if (n >= (1ull << 34) || first_element >= (1ull << 34) || first_element + n >= (1ull << 34))
         return DQ_ERR_UNSUPPORTED;
     if (!out_avg) return DQ_ERR_INVALID_ARG;
-    if (any_nested && !running && !side_info) return DQ_ERR_INVALID_ARG;
+    if (side_first && msgs[0].kind != DQ_KIND_DQSG) return DQ_ERR_INVALID_ARG;   // message 0 is decoded on its own
+    if (any_nested && !running && !side_first && !side_info) return DQ_ERR_INVALID_ARG;
     if (!aligned16(out_avg) || (side_info && !aligned16(side_info))) return DQ_ERR_ALIGNMENT;
     for (uint32_t w = 0; w < W; ++w) {
         if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
         if (!aligned16(msgs[w].packed) || !aligned16(msgs[w].scale)) return DQ_ERR_ALIGNMENT;
     }
-    const bool reads_side = any_nested && !running;
+    const bool reads_side = any_nested && !running && !side_first;
+    const bool from_first = any_nested && !running && side_first;
     a.side = reads_side ? virtual_base(side_info, first_element) : nullptr;
     a.out = virtual_base(out_avg, first_element);
     a.status = status_word;
@@ -375,6 +378,8 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
     if (half_dithered) le = dq::launch_decode_d0_r0(side_map, out_map, a, sms, st);
     else if (running && any_nested) le = d16 ? dq::launch_decode_d16_r1(side_map, out_map, a, sms, st)
                                              : dq::launch_decode_d32_r1(side_map, out_map, a, sms, st);
+    else if (from_first) le = d16 ? dq::launch_decode_d16_r2(side_map, out_map, a, sms, st)
+                                  : dq::launch_decode_d32_r2(side_map, out_map, a, sms, st);
     else le = d16 ? dq::launch_decode_d16_r0(side_map, out_map, a, sms, st)
                   : dq::launch_decode_d32_r0(side_map, out_map, a, sms, st);
     if (le != cudaSuccess) return DQ_ERR_CUDA;
@@ -430,6 +435,13 @@ dq_status ndqsg_decode_aggregate(const dq_msg* msgs, uint32_t W, uint64_t n, uin
 {
     return decode_common(msgs, W, n, step, side_info, out_avg, status_word, true,
                          static_cast<cudaStream_t>(cuda_stream));
+}
+
+dq_status ndqsg_decode_aggregate_side_first(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, float* out_avg,
+                                            uint32_t* status_word, void* cuda_stream)
+{
+    return decode_common(msgs, W, n, step, nullptr, out_avg, status_word, true,
+                         static_cast<cudaStream_t>(cuda_stream), false, false, 0u, true);
 }
 
 dq_status dqsg_decode_aggregate_half_dithered(const dq_msg* msgs, uint32_t W, uint64_t n, float* out_avg,

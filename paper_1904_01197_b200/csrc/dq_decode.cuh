@@ -24,6 +24,10 @@
 
 namespace dq {
 
+// Where the side information of the nested messages comes from: a vector given by the caller (or none at all: only
+// DQSG messages), the running mean of the messages decoded so far, or the reconstruction of message 0.
+enum DecSide : int { kSideGiven = 0, kSideRunning = 1, kSideFirst = 2 };
+
 enum DecKind : uint32_t { kDecDqsg = 0, kDecNdqsgPow2 = 1, kDecNdqsgPow2Shrink = 2, kDecNdqsgAnyK = 3 };
 
 struct DecWorker {
@@ -223,14 +227,16 @@ __device__ __forceinline__ void decode_row_variant(const DecWorker& wk, uint32_t
 
 // The last row of a gradient whose length is not a multiple of 32: one element at a time, everything at run
 // time, straight from and to global memory.  Same arithmetic, in the same order, as decode_row.
-template <int DITH, bool RUN>
+template <int DITH, int SIDE>
 __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint32_t row, uint32_t bucket, uint32_t nvalid)
 {
+    constexpr bool RUN = (SIDE == kSideRunning);
     for (uint32_t e = 0; e < nvalid; ++e) {
         const uint64_t i = (uint64_t)row * 32u + e;
-        const float yside = (!RUN && args.has_side) ? __ldg(args.side + i) : 0.0f;
+        float yside = (!RUN && args.has_side) ? __ldg(args.side + i) : 0.0f;
         float acc = 0.0f;
         for (uint32_t w = 0; w < args.W; ++w) {
+            if (SIDE == kSideFirst && w == 1u) yside = acc;      // the reconstruction of message 0
             const DecWorker& wk = args.w[w];
             const uint32_t kind = wk.variant >> 3;
             const uint32_t bits = wk.bits;
@@ -281,11 +287,12 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint32_t
 // side_map / out_map: [whole rows x 32 floats] views of the caller's side information and output (valid when
 // args.use_tiles; side_map only when args.has_side).
 // ---------------------------------------------------------------------------------------------------
-template <int DITH, bool RUN>
+template <int DITH, int SIDE>
 __global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
 decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __grid_constant__ CUtensorMap out_map,
                         const __grid_constant__ DecodeArgs args)
 {
+    constexpr bool RUN = (SIDE == kSideRunning);
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_side_mem[kDecWarps][kDecTileBuffers];
 
@@ -296,7 +303,7 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t tiles = smem_base + warp * (uint32_t)(kDecTileBuffers * kDecTileBytes);
     const uint32_t bar_side = smem_u32(&bar_side_mem[warp][0]);
-    const bool side_tiles = !RUN && args.has_side != 0u && args.use_tiles != 0u;
+    const bool side_tiles = SIDE == kSideGiven && args.has_side != 0u && args.use_tiles != 0u;
 
     if (lane == 0) {
 #pragma unroll
@@ -386,6 +393,16 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
                 kappa_next = (w + 1u < args.W) ? __ldg(args.w[w + 1u].scale + bucket)
                                                : __ldg(args.w[0].scale + bucket_next);
                 decode_row_variant<DITH, RUN>(args.w[w], row, load_row, kappa, row_addr, acc, args.half_bias_bits);
+                if (SIDE == kSideFirst && w == 0u) {
+                    // the accumulators are now the reconstruction of message 0: it is the side information of
+                    // the nested messages that follow, which read it from the lane's row of the tile buffer
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
+                                     ::"r"(row_addr ^ (uint32_t)(c << 4)), "f"(acc[4 * c]), "f"(acc[4 * c + 1]),
+                                       "f"(acc[4 * c + 2]), "f"(acc[4 * c + 3])
+                                     : "memory");
+                }
                 const uint32_t kb = __float_as_uint(kappa) & 0x7FFFFFFFu;
                 kappa_bits_max = (kb > kappa_bits_max) ? kb : kappa_bits_max;
             }
@@ -413,7 +430,7 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
         }
         if (args.status != nullptr && kappa_bits_max >= 0x7F800000u && row < args.full_rows) atomicOr(args.status, 0x1u);
         if (row == args.full_rows && row < args.rows)
-            decode_partial_row<DITH, RUN>(args, row, bucket_of(row), (uint32_t)(args.n - (uint64_t)row * 32u));
+            decode_partial_row<DITH, SIDE>(args, row, bucket_of(row), (uint32_t)(args.n - (uint64_t)row * 32u));
     }
     // shared memory must stay valid until the last stores have read it
     if (lane == 0) bulk_wait_group_read<0>();

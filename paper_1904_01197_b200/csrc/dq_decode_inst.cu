@@ -1,12 +1,12 @@
 // Instantiation of decode_aggregate_kernel for one dither width and one side-information mode (DQ_INST_DITH,
-// DQ_INST_RUN, given on the compiler's command line).
+// DQ_INST_RUN = a DecSide value, given on the compiler's command line).
 #include <atomic>
 
 #include "dq_decode.cuh"
 #include "dq_launch.h"
 
 #ifndef DQ_INST_DITH
-#error "compile with -DDQ_INST_DITH=<32|16|0> -DDQ_INST_RUN=<0|1>"
+#error "compile with -DDQ_INST_DITH=<32|16|0> -DDQ_INST_RUN=<0|1|2>"
 #endif
 
 namespace dq {
@@ -17,7 +17,7 @@ namespace dq {
 cudaError_t DQ_NAME(DQ_INST_DITH, DQ_INST_RUN)(const CUtensorMap& side_map, const CUtensorMap& out_map,
                                                const DecodeArgs& a, int sm_count, cudaStream_t st)
 {
-    auto k = decode_aggregate_kernel<DQ_INST_DITH, (DQ_INST_RUN != 0)>;
+    auto k = decode_aggregate_kernel<DQ_INST_DITH, DQ_INST_RUN>;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     // per device: the shared-memory attribute and the resident CTAs per SM

@@ -44,12 +44,14 @@ DQ_DECLARE_ENCODE(0, 32) DQ_DECLARE_ENCODE(1, 32) DQ_DECLARE_ENCODE(2, 32) DQ_DE
 DQ_DECLARE_ENCODE(0, 16) DQ_DECLARE_ENCODE(1, 16) DQ_DECLARE_ENCODE(2, 16) DQ_DECLARE_ENCODE(3, 16)
 #undef DQ_DECLARE_ENCODE
 
-// Decoder: dith = 32, 16 or 0 (no dither at the receiver); run = side information is the running mean.
+// Decoder: dith = 32, 16 or 0 (no dither at the receiver); run = DecSide (0 given vector or none, 1 running mean,
+// 2 reconstruction of message 0).
 // The grid (persistent CTAs) follows from a.num_units and the device.
 #define DQ_DECLARE_DECODE(DITH, RUN)                                                                               \
     cudaError_t launch_decode_d##DITH##_r##RUN(const CUtensorMap& side_map, const CUtensorMap& out_map,            \
                                                const DecodeArgs& a, int sm_count, cudaStream_t st);
 DQ_DECLARE_DECODE(32, 0) DQ_DECLARE_DECODE(32, 1) DQ_DECLARE_DECODE(16, 0) DQ_DECLARE_DECODE(16, 1)
+DQ_DECLARE_DECODE(32, 2) DQ_DECLARE_DECODE(16, 2)
 DQ_DECLARE_DECODE(0, 0)
 #undef DQ_DECLARE_DECODE
 
