@@ -162,10 +162,16 @@ class Message:
         return DqMsg(pk, sc, self.seed, self.worker, self.kind, self.params)
 
 
+def new_output(numel: int, dtype, device) -> torch.Tensor:
+    """Every output tensor that this binding allocates on behalf of the caller comes from here (one place to
+    hook, e.g. for tests that surround outputs with guard words)."""
+    return torch.empty(numel, dtype=dtype, device=device)
+
+
 def alloc_message(n: int, params: DqParams, device="cuda"):
     """Uninitialised output buffers for one encode call (packed words as int32, scales as fp32)."""
-    packed = torch.empty(max(1, packed_words(n, params.bits)), dtype=torch.int32, device=device)
-    scale = torch.empty(max(1, num_buckets(n, params.bucket)), dtype=torch.float32, device=device)
+    packed = new_output(max(1, packed_words(n, params.bits)), torch.int32, device)
+    scale = new_output(max(1, num_buckets(n, params.bucket)), torch.float32, device)
     return packed, scale
 
 
@@ -248,7 +254,7 @@ def _msg_array(msgs: Sequence[Message], host: bool = False):
 def dqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, out_avg: Optional[torch.Tensor] = None,
                           stream=None) -> torch.Tensor:
     if out_avg is None:
-        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+        out_avg = new_output(max(1, n), torch.float32, msgs[0].packed.device)
     _check(lib().dqsg_decode_aggregate(_msg_array(msgs), len(msgs), n, step,
                                        _dev_ptr(out_avg, torch.float32, "out_avg"), _stream_ptr(stream)),
            "dqsg_decode_aggregate")
@@ -259,7 +265,7 @@ def ndqsg_decode_aggregate(msgs: Sequence[Message], n: int, step: int, side_info
                            out_avg: Optional[torch.Tensor] = None, status_word: Optional[torch.Tensor] = None,
                            stream=None) -> torch.Tensor:
     if out_avg is None:
-        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+        out_avg = new_output(max(1, n), torch.float32, msgs[0].packed.device)
     _check(lib().ndqsg_decode_aggregate(_msg_array(msgs), len(msgs), n, step,
                                         _dev_ptr(side_info, torch.float32, "side_info"),
                                         _dev_ptr(out_avg, torch.float32, "out_avg"),
@@ -273,7 +279,7 @@ def ndqsg_decode_aggregate_range(msgs: Sequence[Message], n: int, first_element:
                                  status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """Fused decode-and-average of a bucket range: every buffer holds the range's data only."""
     if out_avg is None:
-        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+        out_avg = new_output(max(1, n), torch.float32, msgs[0].packed.device)
     _check(lib().ndqsg_decode_aggregate_range(_msg_array(msgs), len(msgs), n, first_element, step,
                                               _dev_ptr(side_info, torch.float32, "side_info"),
                                               _dev_ptr(out_avg, torch.float32, "out_avg"),
@@ -286,7 +292,7 @@ def dqsg_decode_aggregate_half_dithered(msgs: Sequence[Message], n: int, out_avg
                                         stream=None) -> torch.Tensor:
     """Mean of the DQSG messages reconstructed without subtracting the dither (Section 2.1, Lemma 1)."""
     if out_avg is None:
-        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+        out_avg = new_output(max(1, n), torch.float32, msgs[0].packed.device)
     _check(lib().dqsg_decode_aggregate_half_dithered(_msg_array(msgs), len(msgs), n,
                                                      _dev_ptr(out_avg, torch.float32, "out_avg"),
                                                      _stream_ptr(stream)), "dqsg_decode_aggregate_half_dithered")
@@ -298,7 +304,7 @@ def ndqsg_decode_aggregate_running(msgs: Sequence[Message], n: int, step: int,
                                    status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """Algorithm 2's server loop: NDQSG messages are decoded against the mean of the messages before them."""
     if out_avg is None:
-        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+        out_avg = new_output(max(1, n), torch.float32, msgs[0].packed.device)
     _check(lib().ndqsg_decode_aggregate_running(_msg_array(msgs), len(msgs), n, step,
                                                 _dev_ptr(out_avg, torch.float32, "out_avg"),
                                                 _dev_ptr(status_word, torch.int32, "status_word"),
@@ -311,7 +317,7 @@ def ndqsg_decode_aggregate_side_first(msgs: Sequence[Message], n: int, step: int
                                       status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """Algorithm 2 with one P1 worker: the reconstruction of message 0 is the side information of the rest."""
     if out_avg is None:
-        out_avg = torch.empty(max(1, n), dtype=torch.float32, device=msgs[0].packed.device)
+        out_avg = new_output(max(1, n), torch.float32, msgs[0].packed.device)
     _check(lib().ndqsg_decode_aggregate_side_first(_msg_array(msgs), len(msgs), n, step,
                                                    _dev_ptr(out_avg, torch.float32, "out_avg"),
                                                    _dev_ptr(status_word, torch.int32, "status_word"),
@@ -323,7 +329,7 @@ def code_histogram(packed: torch.Tensor, n: int, bits: int, hist: Optional[torch
                    stream=None) -> torch.Tensor:
     """hist[c] = number of elements of the packed message whose code is c (int64[2^bits] on the device)."""
     if hist is None:
-        hist = torch.empty(1 << bits, dtype=torch.int64, device=packed.device)
+        hist = new_output(1 << bits, torch.int64, packed.device)
     _check(lib().dq_code_histogram(_dev_ptr(packed, torch.int32, "packed"), n, bits,
                                    _dev_ptr(hist, torch.int64, "hist"), _stream_ptr(stream)), "dq_code_histogram")
     return hist
@@ -346,7 +352,7 @@ def ternary_pack(packed: torch.Tensor, n: int, out: Optional[torch.Tensor] = Non
                  status_word: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """2-bit stream of a three-level message -> five codes per byte (uint8[ternary_bytes(n)] on the device)."""
     if out is None:
-        out = torch.empty(max(1, ternary_bytes(n)), dtype=torch.uint8, device=packed.device)
+        out = new_output(max(1, ternary_bytes(n)), torch.uint8, packed.device)
     _check(lib().dq_ternary_pack(_dev_ptr(packed, torch.int32, "packed"), n, _dev_ptr(out, torch.uint8, "out"),
                                  _dev_ptr(status_word, torch.int32, "status_word"), _stream_ptr(stream)),
            "dq_ternary_pack")
@@ -356,7 +362,7 @@ def ternary_pack(packed: torch.Tensor, n: int, out: Optional[torch.Tensor] = Non
 def ternary_unpack(data: torch.Tensor, n: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """Five codes per byte -> the 2-bit stream (int32[packed_words(n, 2)] on the device)."""
     if out is None:
-        out = torch.empty(max(1, packed_words(n, 2)), dtype=torch.int32, device=data.device)
+        out = new_output(max(1, packed_words(n, 2)), torch.int32, data.device)
     _check(lib().dq_ternary_unpack(_dev_ptr(data, torch.uint8, "data"), n, _dev_ptr(out, torch.int32, "out"),
                                    _stream_ptr(stream)), "dq_ternary_unpack")
     return out

@@ -35,3 +35,63 @@ def pytest_collection_modifyitems(config, items):
 @pytest.fixture(scope="session")
 def golden_dir():
     return GOLDEN
+
+
+GUARD_BYTES = 256
+CURRENT_GUARD = None        # the GuardedOutputs of the GPU test that is running
+GUARD_PATTERN = 0xA5
+
+
+class GuardedOutputs:
+    """Stands in for the out-of-bounds checker of a sanitizer: every output buffer that the binding allocates is
+    carved out of a larger one with GUARD_BYTES of a known pattern before and after it, and the pattern is checked
+    when the test ends.  A kernel that writes one byte past (or before) an output fails the test that ran it."""
+
+    def __init__(self, torch):
+        self.torch = torch
+        self.buffers = []
+
+    def new_output(self, numel, dtype, device):
+        torch = self.torch
+        nbytes = numel * torch.empty((), dtype=dtype).element_size()
+        padded = (nbytes + 15) // 16 * 16                     # the view must keep 16-byte alignment on both sides
+        buf = torch.full((GUARD_BYTES + padded + GUARD_BYTES,), GUARD_PATTERN, dtype=torch.uint8, device=device)
+        self.buffers.append((buf, nbytes))
+        return buf[GUARD_BYTES:GUARD_BYTES + nbytes].view(dtype)
+
+    def host_output(self, numel, dtype):
+        """The same for a pinned host buffer that a *_host entry point fills."""
+        torch = self.torch
+        nbytes = numel * torch.empty((), dtype=dtype).element_size()
+        padded = (nbytes + 15) // 16 * 16
+        buf = torch.full((GUARD_BYTES + padded + GUARD_BYTES,), GUARD_PATTERN, dtype=torch.uint8).pin_memory()
+        self.buffers.append((buf, nbytes))
+        return buf[GUARD_BYTES:GUARD_BYTES + nbytes].view(dtype)
+
+    def check(self):
+        torch = self.torch
+        if self.buffers and torch.cuda.is_available():
+            torch.cuda.synchronize()
+        for k, (buf, nbytes) in enumerate(self.buffers):
+            front = buf[:GUARD_BYTES]
+            back = buf[GUARD_BYTES + nbytes:]
+            assert bool((front == GUARD_PATTERN).all()), f"output {k} ({nbytes} bytes): bytes before it were overwritten"
+            assert bool((back == GUARD_PATTERN).all()), f"output {k} ({nbytes} bytes): bytes after it were overwritten"
+        self.buffers.clear()
+
+
+@pytest.fixture(autouse=True)
+def guarded_outputs(request, monkeypatch):
+    """GPU tests run with guard words around every output the binding allocates (see GuardedOutputs)."""
+    if "gpu" not in request.keywords or not _have_gpu():
+        yield None
+        return
+    import torch
+    from paper_1904_01197_b200 import binding
+    global CURRENT_GUARD
+    g = GuardedOutputs(torch)
+    monkeypatch.setattr(binding, "new_output", g.new_output)
+    CURRENT_GUARD = g
+    yield g
+    CURRENT_GUARD = None
+    g.check()

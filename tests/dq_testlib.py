@@ -53,3 +53,11 @@ def assert_fp32_close(got: np.ndarray, ref: np.ndarray, what: str = ""):
     bad = err > tol
     assert not bad.any(), f"{what}: {int(bad.sum())} of {bad.size} outside tolerance, worst {err.max()} at {int(err.argmax())}"
     return bool(np.array_equal(got.view(np.uint32), ref.view(np.uint32)))
+
+
+def host_output(torch, numel: int, dtype):
+    """A pinned host buffer for a *_host entry point's output, with guard words around it while a GPU test runs."""
+    import conftest
+    if conftest.CURRENT_GUARD is not None:
+        return conftest.CURRENT_GUARD.host_output(numel, dtype)
+    return torch.empty(numel, dtype=dtype).pin_memory()

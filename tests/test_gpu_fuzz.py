@@ -10,7 +10,7 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
-from dq_testlib import assert_fp32_close  # noqa: E402
+from dq_testlib import assert_fp32_close, host_output  # noqa: E402
 from test_gpu_parity import _check_encode, _roundtrip_decode, dq, oracle  # noqa: E402,F401
 
 BUCKETS = [32, 64, 96, 160, 256, 480, 512, 1024, 1504, 2048, 4096, 8192, 12288]
@@ -83,8 +83,8 @@ def test_random_host_buffer_round_trip(dq, oracle, case):
     host_msgs, omsgs = [], []
     for w, (g, sp) in enumerate(zip(grads, specs)):
         p = spec_params(dq, sp, bucket)
-        pk = torch.empty(max(1, dq.packed_words(n, sp.bits)), dtype=torch.int32).pin_memory()
-        sc = torch.empty(max(1, dq.num_buckets(n, bucket)), dtype=torch.float32).pin_memory()
+        pk = host_output(torch, max(1, dq.packed_words(n, sp.bits)), torch.int32)
+        sc = host_output(torch, max(1, dq.num_buckets(n, bucket)), torch.float32)
         ws = torch.empty(dq.encode_workspace_bytes(n, p), dtype=torch.uint8, device="cuda")
         fn = dq.dqsg_encode_host if sp.kind == DQSG else dq.ndqsg_encode_host
         fn(torch.from_numpy(g).pin_memory(), sp.seed, w, step, p, pk, sc, ws)
@@ -94,7 +94,7 @@ def test_random_host_buffer_round_trip(dq, oracle, case):
         host_msgs.append(dq.Message(pk, sc, sp.seed, w, sp.kind, p))
         omsgs.append(oracle_msg(oracle, opk, osc, sp, w, bucket))
     any_nd = any(s.kind == NDQSG for s in specs)
-    out = torch.empty(n, dtype=torch.float32).pin_memory()
+    out = host_output(torch, n, torch.float32)
     ws = torch.empty(dq.decode_workspace_bytes(host_msgs, n, any_nd), dtype=torch.uint8, device="cuda")
     dq.ndqsg_decode_aggregate_host(host_msgs, n, step, torch.from_numpy(side).pin_memory() if any_nd else None, out, ws)
     ref = oracle.decode_aggregate(omsgs, n, step, side_info=side if any_nd else None, threads=4)

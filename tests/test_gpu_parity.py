@@ -28,7 +28,8 @@ def oracle():
     return oracle
 
 
-from dq_testlib import (assert_fp32_close, gpu_encode, gpu_msg, oracle_encode, oracle_msg, words_np)  # noqa: E402
+from dq_testlib import (assert_fp32_close, gpu_encode, gpu_msg, host_output, oracle_encode, oracle_msg,  # noqa: E402
+                        words_np)
 
 
 def _specs_for_bits(bits):
@@ -243,8 +244,8 @@ def test_host_buffer_entry_points(dq, oracle):
         p = dq.binding.make_params(bucket, sp.bits, sp.levels, sp.coarse_K, sp.fine_M, sp.alpha)
         ws = torch.empty(dq.encode_workspace_bytes(n, p), dtype=torch.uint8, device="cuda")
         gh = torch.from_numpy(g).pin_memory()
-        pk = torch.empty(dq.packed_words(n, sp.bits), dtype=torch.int32).pin_memory()
-        sc = torch.empty(dq.num_buckets(n, bucket), dtype=torch.float32).pin_memory()
+        pk = host_output(torch, dq.packed_words(n, sp.bits), torch.int32)
+        sc = host_output(torch, dq.num_buckets(n, bucket), torch.float32)
         fn = dq.dqsg_encode_host if sp.kind == DQSG else dq.ndqsg_encode_host
         fn(gh, sp.seed, w, 4, p, pk, sc, ws)
         opk, osc = oracle_encode(oracle, g, sp, w, 4, bucket)
@@ -252,7 +253,7 @@ def test_host_buffer_entry_points(dq, oracle):
         msgs.append(dq.Message(pk, sc, sp.seed, w, sp.kind, p))
         omsgs.append(oracle_msg(oracle, opk, osc, sp, w, bucket))
     side = torch.from_numpy((g + 0.01 * rng.standard_normal(n)).astype(np.float32)).pin_memory()
-    out = torch.empty(n, dtype=torch.float32).pin_memory()
+    out = host_output(torch, n, torch.float32)
     ws = torch.empty(dq.decode_workspace_bytes(msgs, n, True), dtype=torch.uint8, device="cuda")
     dq.ndqsg_decode_aggregate_host(msgs, n, 4, side, out, ws)
     ref = oracle.decode_aggregate(omsgs, n, 4, side_info=side.numpy())

@@ -11,8 +11,8 @@ pytestmark = pytest.mark.gpu
 
 torch = pytest.importorskip("torch")
 
-from dq_testlib import (assert_fp32_close, gpu_encode, gpu_msg, oracle_encode, oracle_msg, spec_params,  # noqa: E402
-                        words_np)
+from dq_testlib import (assert_fp32_close, gpu_encode, gpu_msg, host_output, oracle_encode, oracle_msg,  # noqa: E402
+                        spec_params, words_np)
 from test_gpu_parity import dq, oracle  # noqa: E402,F401
 
 SPECS = [WorkerSpec(DQSG, 2, 3, seed=601), WorkerSpec(DQSG, 3, 5, seed=602), WorkerSpec(DQSG, 1, 2, seed=603),
@@ -138,7 +138,7 @@ def test_host_buffer_decode_of_a_long_gradient(dq, oracle, bucket, bits_mix):
         host_msgs.append(dq.Message(hpk, hsc, sp.seed, w, sp.kind, spec_params(dq, sp, bucket)))
         keep += [pk, sc, hpk, hsc]
     whole = dq.ndqsg_decode_aggregate(dev_msgs, n, step, torch.from_numpy(side).cuda())[:n].cpu().numpy()
-    out = torch.empty(n, dtype=torch.float32).pin_memory()
+    out = host_output(torch, n, torch.float32)
     ws = torch.empty(dq.decode_workspace_bytes(host_msgs, n, True), dtype=torch.uint8, device="cuda")
     for _ in range(2):                                   # twice: the staging area is reused
         out.zero_()
