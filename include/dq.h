@@ -23,10 +23,18 @@
  *   - A message is `scale` (one fp32 per bucket) plus `packed`: element i's b-bit code at bit offset
  *     i*b of a little-endian stream of 32-bit words; pad bits of the last word are written as 0.
  *   - "device" pointers are CUDA device memory on the current device, 16-byte aligned, owned by the
- *     caller.  The library allocates nothing, keeps no state between calls, and is asynchronous on the
- *     given stream (it never synchronises), except for the *_host entry points, which return after the
- *     results are in the caller's host buffers.
+ *     caller.  The library allocates nothing at run time and keeps no state between calls, with two
+ *     exceptions that live in its device image: one error word per GPU (dq_device_error_flags) and the
+ *     fixed staging array of dqsg_encode_host_static.  It is asynchronous on the given stream (it never
+ *     synchronises), except for the *_host entry points, which return after the results are in the
+ *     caller's host buffers.
  *   - Outputs must not alias inputs.  Inputs are assumed finite.
+ *   - The integer decisions are taken in fp32 with the rounding constant 1.5 * 2^23, which is exact for
+ *     magnitudes below 2^22: DQSG needs (L-1)/2 + 1 < 2^22 (always true for b <= 8); NDQSG needs
+ *     alpha*M1 <= 2^20 (checked) and, at the decoder, |alpha*M1*y/kappa| < 2^21 for every element, i.e. side
+ *     information that is not millions of coarse cells away from the gradient -- in particular a message
+ *     whose bucket scale kappa is almost zero (below about 1e-6 of |y|) must not be paired with ordinary
+ *     side information.  Beyond that bound the resolved coset is undefined (no fault, no diagnostic).
  *   - Errors are return codes only.  Invalid arguments are rejected before anything is launched.
  *   - n must be below 2^34.
  */
@@ -89,6 +97,14 @@ typedef struct {
  * one still sees both complete.  Results are identical with and without the flag.
  */
 #define DQ_FLAG_OUTPUT_FREE 0x2u
+/*
+ * DQ_FLAG_TEST_DROP_COPY (encoders only; for tests of the error path, never for production calls).  One warp
+ * of the encoder announces the tile copy of its last work unit but does not issue it.  Its bounded wait for
+ * that copy runs out after about 20 ms; the kernel then finishes normally, DQ_ERR_COPY_TIMEOUT is set in the
+ * device's error word (dq_device_error_flags) and the codes of that one unit are undefined.  Nothing faults
+ * and nothing waits longer than the bound.  Without effect for gradients so short that the warp has one unit.
+ */
+#define DQ_FLAG_TEST_DROP_COPY 0x80000000u
 
 /* One worker's message as the decoder sees it. */
 typedef struct {
@@ -222,6 +238,16 @@ dq_status ndqsg_decode_aggregate_range(const dq_msg* msgs, uint32_t W, uint64_t 
 dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, uint64_t* hist, void* cuda_stream);
 
 /*
+ * dq_code_entropy -- the empirical entropy H = -sum_c p_c log2 p_c, p_c = hist[c] / sum(hist), of a code
+ * histogram, in bits per element: the rate that the entropy coding of the index stream approaches (Section 4,
+ * the paragraph on entropy coding and the entropy-coded columns of the tables).  Host arithmetic on at most 256
+ * counters.
+ *   hist_host             HOST memory, uint64[2^bits] (a copy of dq_code_histogram's result)
+ *   out_bits_per_element  HOST, receives H; 0 for an empty histogram
+ */
+dq_status dq_code_entropy(const uint64_t* hist_host, uint32_t bits, double* out_bits_per_element);
+
+/*
  * Radix-3 container for three-level DQSG messages (levels = 3, bits = 2).  Section 4 counts log2(3) = 1.585
  * bits per element for the three-level quantizer (raw-bits table, DQSGD row); the 2-bit stream spends 2.  The
  * container stores five codes per byte,
@@ -278,9 +304,13 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
  *   returns DQ_ERR_TOO_LARGE      when dq_encode_workspace_bytes(n, p) > DQ_STATIC_SCRATCH_BYTES
  *                                 (about 7.8 million elements at 2 bits); nothing is copied or launched
  *
- * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.  The first call on
- * each device looks up the array's device address (once per device, with that device current); make that
- * first call outside any stream capture.  The array is shared by all calls and keeps whatever the last call
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.  The array is part of
+ * the library's device image: the driver reserves it when that image is loaded on a device, which with lazy
+ * loading is the first use of ANY entry point there; if the memory cannot be reserved, every entry point fails
+ * with DQ_ERR_CUDA.  The first call of this function on each device additionally looks up the array's device
+ * address (once per device, with that device current); make one warm-up call per device at start-up, outside
+ * any stream capture and outside the latency-critical loop.  The address is cached for the life of the
+ * process: cudaDeviceReset is not supported once it has been looked up.  The array is shared by all calls and keeps whatever the last call
  * left in it.  Nothing in it has to start at zero: the gradient is copied over its input region and the
  * kernel writes every packed word and every scale before they are copied back.  Two calls that overlap in
  * time on one device (different host threads or streams) use the same bytes and race; serialise them.

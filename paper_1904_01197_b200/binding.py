@@ -20,6 +20,7 @@ DQ_ERR_COPY_TIMEOUT = 0x2
 DQ_WARN_CODE_RANGE = 0x4
 DQ_FLAG_INPUT_READY = 0x1
 DQ_FLAG_OUTPUT_FREE = 0x2
+DQ_FLAG_TEST_DROP_COPY = 0x80000000
 
 _LIB_PATH = Path(__file__).resolve().parent / "lib" / "libdq_b200.so"
 
@@ -73,6 +74,8 @@ def lib() -> C.CDLL:
         L.ndqsg_decode_aggregate_side_first.restype = C.c_int
         L.dq_code_histogram.argtypes = [vp, u64, u32, vp, vp]
         L.dq_code_histogram.restype = C.c_int
+        L.dq_code_entropy.argtypes = [C.POINTER(C.c_uint64), u32, C.POINTER(C.c_double)]
+        L.dq_code_entropy.restype = C.c_int
         for f in (L.dqsg_encode_range, L.ndqsg_encode_range):
             f.argtypes = [vp, u64, u64, u64, u32, u64, pp, vp, vp, vp]; f.restype = C.c_int
         L.ndqsg_decode_aggregate_range.argtypes = [pm, u32, u64, u64, u64, vp, vp, vp, vp]
@@ -336,11 +339,13 @@ def code_histogram(packed: torch.Tensor, n: int, bits: int, hist: Optional[torch
 
 
 def entropy_bits_per_element(hist) -> float:
-    """Empirical entropy -sum p log2 p of a code histogram (host arithmetic on at most 256 counters)."""
-    import math
+    """Empirical entropy of a code histogram in bits per element (dq_code_entropy on a host copy of it)."""
     counts = [int(c) for c in hist.tolist()]
-    total = sum(counts)
-    return -sum(c / total * math.log2(c / total) for c in counts if c) if total else 0.0
+    bits = max(1, (len(counts) - 1).bit_length())
+    arr = (C.c_uint64 * (1 << bits))(*counts)
+    out = C.c_double(0.0)
+    _check(lib().dq_code_entropy(arr, bits, C.byref(out)), "dq_code_entropy")
+    return float(out.value)
 
 
 # ------------------------------------------------------------------------------------------ radix-3 container

@@ -3,6 +3,7 @@
 #include "dq.h"
 
 #include <atomic>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <utility>
@@ -212,6 +213,7 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
     fill_philox(a.ps, seed, worker, step);
     a.early_read = (p->flags & DQ_FLAG_INPUT_READY) ? 1u : 0u;
     a.early_store = (a.early_read && (p->flags & DQ_FLAG_OUTPUT_FREE)) ? 1u : 0u;
+    a.test_drop_copy = (p->flags & DQ_FLAG_TEST_DROP_COPY) ? 1u : 0u;
     a.error_flags = error_flags_address();
     if (!a.error_flags) return DQ_ERR_CUDA;
 
@@ -506,6 +508,23 @@ dq_status dq_code_histogram(const uint32_t* packed, uint64_t n, uint32_t bits, u
     return DQ_OK;
 }
 
+dq_status dq_code_entropy(const uint64_t* hist_host, uint32_t bits, double* out_bits_per_element)
+{
+    if (!hist_host || !out_bits_per_element || bits < 1u || bits > 8u) return DQ_ERR_INVALID_ARG;
+    long double total = 0.0L;
+    for (uint32_t c = 0; c < (1u << bits); ++c) total += (long double)hist_host[c];
+    long double h = 0.0L;
+    if (total > 0.0L) {
+        for (uint32_t c = 0; c < (1u << bits); ++c) {
+            if (hist_host[c] == 0u) continue;
+            const long double pc = (long double)hist_host[c] / total;
+            h -= pc * log2l(pc);
+        }
+    }
+    *out_bits_per_element = (double)h;
+    return DQ_OK;
+}
+
 // ------------------------------------------------------------------------------------------------ radix-3 container
 uint64_t dq_ternary_bytes(uint64_t n) { return (n + 4u) / 5u; }
 
@@ -571,6 +590,7 @@ static dq_status encode_host(dq_kind kind, const float* grad, uint64_t n, uint64
     dq_status s = check_params(p, kind, &L, &alpha);
     if (s != DQ_OK) return s;
     if (n == 0) return DQ_OK;
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
     if (!grad || !out_packed || !out_scale || !workspace) return DQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0u) return DQ_ERR_ALIGNMENT;
     if (workspace_bytes < dq_encode_workspace_bytes(n, p)) return DQ_ERR_INVALID_ARG;
@@ -585,7 +605,10 @@ static dq_status encode_host(dq_kind kind, const float* grad, uint64_t n, uint64
     const uint64_t sbytes = dq_num_buckets(n, p->bucket) * 4u;
     if (cudaMemcpyAsync(d_grad, grad, n * 4u, cudaMemcpyHostToDevice, st) != cudaSuccess) return DQ_ERR_CUDA;
     s = encode_common(kind, d_grad, n, seed, worker, step, p, d_packed, d_scale, st);
-    if (s != DQ_OK) return s;
+    if (s != DQ_OK) {
+        cudaStreamSynchronize(st);          // the copy above may still be reading the caller's buffer
+        return s;
+    }
     if (cudaMemcpyAsync(out_packed, d_packed, pbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaMemcpyAsync(out_scale, d_scale, sbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
@@ -619,8 +642,13 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
         dq_status s = check_params(&msgs[w].p, msgs[w].kind, &L, &alpha);
         if (s != DQ_OK) return s;
         if (!msgs[w].packed || !msgs[w].scale) return DQ_ERR_INVALID_ARG;
+        // what decode_common would reject, checked here before any copy is queued
+        if (msgs[w].p.bucket != msgs[0].p.bucket) return DQ_ERR_UNSUPPORTED;
+        if ((msgs[w].p.dither_bits == 16u) != (msgs[0].p.dither_bits == 16u)) return DQ_ERR_UNSUPPORTED;
+        if (msgs[w].kind == DQ_KIND_NDQSG && !side_info) return DQ_ERR_INVALID_ARG;
     }
     if (n == 0) return DQ_OK;
+    if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
     if (!out_avg || !workspace) return DQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0u) return DQ_ERR_ALIGNMENT;
     if (workspace_bytes < dq_decode_workspace_bytes(msgs, W, n, side_info != nullptr)) return DQ_ERR_INVALID_ARG;
@@ -649,7 +677,10 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
         dev_msgs[w].scale = d_s;
     }
     dq_status s = decode_common(dev_msgs, W, n, step, d_side, d_out, nullptr, true, st);
-    if (s != DQ_OK) return s;
+    if (s != DQ_OK) {
+        cudaStreamSynchronize(st);          // copies queued above may still be reading the caller's buffers
+        return s;
+    }
     if (cudaMemcpyAsync(out_avg, d_out, n * 4u, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;

@@ -81,6 +81,8 @@ struct EncodeArgs {
                              // drains, and only its stores wait for it
     uint32_t early_store;    // ... and that the previous kernel neither reads nor writes this call's outputs: nothing
                              // waits for that kernel except the end of this one (see encode_kernel)
+    uint32_t test_drop_copy; // test hook: warp 0 of the first tile CTA arms the barrier for its last unit without
+                             // issuing the copy, so that the bounded wait for it runs out (see DQ_FLAG_TEST_DROP_COPY)
     unsigned int* error_flags;     // the library's per-device error word
     PhiloxStream ps;
 };
@@ -485,8 +487,11 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
                     const uint32_t next = pair + stride;
                     if (next < args.num_units) {
                         mbar_expect_tx(my_bar + 8u * half, (uint32_t)kWarpTileBytes);
-                        tma_load_rows(my_smem + half * kWarpTileBytes, &tmap, my_bar + 8u * half,
-                                      (int32_t)((next * wpb + sub) * 64u + half * 32u));
+                        const bool drop = args.test_drop_copy != 0u && blockIdx.x == args.plain_ctas && warp == 0u &&
+                                          half == 0u && next + stride >= args.num_units;
+                        if (!drop)
+                            tma_load_rows(my_smem + half * kWarpTileBytes, &tmap, my_bar + 8u * half,
+                                          (int32_t)((next * wpb + sub) * 64u + half * 32u));
                     }
                 }
                 const float a = bucket_gain(args.gain_num, mx);
@@ -535,8 +540,10 @@ encode_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ 
             const uint64_t next = tile + (uint64_t)kEncStages * stride;
             if (next < args.num_units) {
                 mbar_expect_tx(my_bar + 8u * s, (uint32_t)kWarpTileBytes);
-                tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s,
-                              (int32_t)(next * 32u));
+                const bool drop = args.test_drop_copy != 0u && blockIdx.x == args.plain_ctas && warp == 0u &&
+                                  next + stride >= args.num_units;
+                if (!drop)
+                    tma_load_rows(my_smem + s * kWarpTileBytes, &tmap, my_bar + 8u * s, (int32_t)(next * 32u));
             }
         }
         const uint32_t row = (uint32_t)tile * 32u + lane;   // row index in the gradient (< 2^29)

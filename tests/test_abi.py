@@ -107,3 +107,25 @@ def test_workspace_sizes(dq):
     need = dq.encode_workspace_bytes(n, p)
     assert need >= n * 4 + dq.packed_words(n, 2) * 4 + dq.num_buckets(n, 2048) * 4
     assert need % 256 == 0
+
+
+def test_host_decode_rejects_bad_message_sets_before_any_copy(dq):
+    """Mixed bucket sizes, mixed dither widths and a nested message without side information are refused by the
+    host-buffer decode before a single byte is copied: every pointer here is a fake that must not be touched."""
+    L = dq.lib()
+    P = dq.binding.make_params
+    fake = 0x1000
+
+    def msg(kind, p):
+        return dq.DqMsg(fake, fake, 1, 0, kind, p)
+
+    def call(msgs, side):
+        arr = (dq.DqMsg * len(msgs))(*msgs)
+        return L.ndqsg_decode_aggregate_host(arr, len(msgs), 4096, 0, side, fake, fake, 1 << 30, None)
+
+    dqsg, nd = dq.DQ_KIND_DQSG, dq.DQ_KIND_NDQSG
+    assert call([msg(dqsg, P(512, 2)), msg(dqsg, P(1024, 2))], None) == 2            # mixed buckets
+    assert call([msg(dqsg, P(512, 2, dither_bits=32)), msg(dqsg, P(512, 2, dither_bits=16))], None) == 2
+    assert call([msg(dqsg, P(512, 2)), msg(nd, P(512, 2, 0, 4, 2.0, 1.0))], None) == 1   # nested, no side info
+    p = P(512, 2)
+    assert L.dqsg_encode_host(fake, 1 << 34, 1, 0, 0, C.byref(p), fake, fake, fake, 1 << 40, None) == 2

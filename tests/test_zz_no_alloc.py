@@ -5,7 +5,8 @@ latency-critical loop that must not call cudaMalloc can still encode: the stagin
 as a fixed device array.  This test drives the entry point through the C ABI with plain numpy buffers (no device
 tensor is created for it), twice in a row with different inputs, because the array is shared between calls and
 keeps the previous call's bytes: the second result must not depend on the first.  The results are compared,
-bit for bit, with `dqsg_encode_host`, which gets its workspace from the caller.
+bit for bit, with `dqsg_encode_host`, which gets its workspace from the caller, and with the CPU oracle's
+encoder, so that the comparison does not rest on the CUDA path alone.
 
 The file is named so that pytest collects it last.
 """
@@ -38,6 +39,13 @@ def _reference(dq, g, seed, worker, step, params):
     return pk.numpy().copy(), sc.numpy().copy()
 
 
+def _oracle(g, seed, worker, step, params):
+    """The CPU oracle's DQSG encoder on the same input."""
+    import oracle
+    oracle.build()
+    return oracle.dqsg_encode(g, seed, worker, step, params.bucket, params.bits, params.levels)
+
+
 def _static(dq, g, seed, worker, step, params):
     """The entry point under test, called straight through ctypes with numpy buffers."""
     n = g.size
@@ -62,6 +70,9 @@ def test_static_scratch_encode_matches_workspace_encode_twice_in_a_row(dq):
         ref_pk, ref_sc = _reference(dq, g, seed, worker, step, params)
         assert np.array_equal(got_sc.view(np.uint32), ref_sc.view(np.uint32))      # scales: bit-exact
         assert np.array_equal(got_pk, ref_pk)                                      # packed words: bit-exact
+        ora_pk, ora_sc = _oracle(g, seed, worker, step, params)
+        assert np.array_equal(got_pk.view(np.uint32), ora_pk), "packed words differ from the oracle's"
+        assert np.array_equal(got_sc.view(np.uint32), ora_sc.view(np.uint32)), "scales differ from the oracle's"
     # and once more with the first input: same answer as before, whatever the array held in between
     g, params, seed, worker, step = cases[0]
     again_pk, again_sc = _static(dq, g, seed, worker, step, params)
