@@ -286,6 +286,10 @@ dq_status ndqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32
 dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
                                       const float* side_info, float* out_avg,
                                       void* workspace, uint64_t workspace_bytes, void* cuda_stream);
+/* ndqsg_decode_aggregate_side_first from host buffers; workspace of dq_decode_workspace_bytes(msgs, W, n, 0). */
+dq_status ndqsg_decode_aggregate_side_first_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                                 float* out_avg, void* workspace, uint64_t workspace_bytes,
+                                                 void* cuda_stream);
 
 /*
  * dqsg_encode_host_static -- dqsg_encode_host for callers that cannot provide device memory.

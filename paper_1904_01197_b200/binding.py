@@ -91,6 +91,8 @@ def lib() -> C.CDLL:
         L.dqsg_encode_host_static.restype = C.c_int
         L.ndqsg_decode_aggregate_host.argtypes = [pm, u32, u64, u64, vp, vp, vp, u64, vp]
         L.ndqsg_decode_aggregate_host.restype = C.c_int
+        L.ndqsg_decode_aggregate_side_first_host.argtypes = [pm, u32, u64, u64, vp, vp, u64, vp]
+        L.ndqsg_decode_aggregate_side_first_host.restype = C.c_int
         L.dq_device_error_flags.argtypes = [C.POINTER(u32)]; L.dq_device_error_flags.restype = C.c_int
         L.dq_launch_count.argtypes = []; L.dq_launch_count.restype = u64
         _lib = L
@@ -423,6 +425,16 @@ def ndqsg_decode_aggregate_host(msgs: Sequence[Message], n: int, step: int, side
                                              _host_ptr(out_avg, torch.float32, "out_avg"),
                                              workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                              _stream_ptr(stream)), "ndqsg_decode_aggregate_host")
+    return out_avg
+
+
+def ndqsg_decode_aggregate_side_first_host(msgs: Sequence[Message], n: int, step: int, out_avg, workspace,
+                                           stream=None):
+    _check(lib().ndqsg_decode_aggregate_side_first_host(_msg_array(msgs, host=True), len(msgs), n, step,
+                                                        _host_ptr(out_avg, torch.float32, "out_avg"),
+                                                        workspace.data_ptr(),
+                                                        workspace.numel() * workspace.element_size(),
+                                                        _stream_ptr(stream)), "ndqsg_decode_aggregate_side_first_host")
     return out_avg
 
 

@@ -631,11 +631,12 @@ dq_status ndqsg_encode_host(const float* grad, uint64_t n, uint64_t seed, uint32
                        workspace_bytes, cuda_stream);
 }
 
-dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
-                                      const float* side_info, float* out_avg, void* workspace,
-                                      uint64_t workspace_bytes, void* cuda_stream)
+static dq_status decode_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step, const float* side_info,
+                             bool side_first, float* out_avg, void* workspace, uint64_t workspace_bytes,
+                             void* cuda_stream)
 {
     if (!msgs || W == 0u || W > DQ_MAX_WORKERS) return DQ_ERR_INVALID_ARG;
+    if (side_first && msgs[0].kind != DQ_KIND_DQSG) return DQ_ERR_INVALID_ARG;
     for (uint32_t w = 0; w < W; ++w) {
         uint32_t L;
         float alpha;
@@ -645,7 +646,7 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
         // what decode_common would reject, checked here before any copy is queued
         if (msgs[w].p.bucket != msgs[0].p.bucket) return DQ_ERR_UNSUPPORTED;
         if ((msgs[w].p.dither_bits == 16u) != (msgs[0].p.dither_bits == 16u)) return DQ_ERR_UNSUPPORTED;
-        if (msgs[w].kind == DQ_KIND_NDQSG && !side_info) return DQ_ERR_INVALID_ARG;
+        if (msgs[w].kind == DQ_KIND_NDQSG && !side_info && !side_first) return DQ_ERR_INVALID_ARG;
     }
     if (n == 0) return DQ_OK;
     if (n >= (1ull << 34)) return DQ_ERR_UNSUPPORTED;
@@ -676,7 +677,7 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
         dev_msgs[w].packed = d_p;
         dev_msgs[w].scale = d_s;
     }
-    dq_status s = decode_common(dev_msgs, W, n, step, d_side, d_out, nullptr, true, st);
+    dq_status s = decode_common(dev_msgs, W, n, step, d_side, d_out, nullptr, true, st, false, false, 0u, side_first);
     if (s != DQ_OK) {
         cudaStreamSynchronize(st);          // copies queued above may still be reading the caller's buffers
         return s;
@@ -684,6 +685,20 @@ dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n
     if (cudaMemcpyAsync(out_avg, d_out, n * 4u, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+dq_status ndqsg_decode_aggregate_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                      const float* side_info, float* out_avg, void* workspace,
+                                      uint64_t workspace_bytes, void* cuda_stream)
+{
+    return decode_host(msgs, W, n, step, side_info, false, out_avg, workspace, workspace_bytes, cuda_stream);
+}
+
+dq_status ndqsg_decode_aggregate_side_first_host(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t step,
+                                                 float* out_avg, void* workspace, uint64_t workspace_bytes,
+                                                 void* cuda_stream)
+{
+    return decode_host(msgs, W, n, step, nullptr, true, out_avg, workspace, workspace_bytes, cuda_stream);
 }
 
 // ------------------------------------------------------------------------------------------------ no allocation

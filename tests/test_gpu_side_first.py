@@ -61,3 +61,23 @@ def test_side_first_needs_a_dqsg_message_first(dq):
     sc = torch.ones(4, dtype=torch.float32, device="cuda")
     with pytest.raises(dq.DqError):
         dq.ndqsg_decode_aggregate_side_first([gpu_msg(dq, pk, sc, sp, 0, 32)], 64, 0)
+
+
+def test_side_first_from_host_buffers(dq, oracle):
+    from dq_testlib import host_output
+    n, bucket, step = 70 * 1024 + 5, 1024, 3
+    rng = np.random.default_rng(99)
+    c = (0.01 * rng.standard_normal(n)).astype(np.float32)
+    specs = [WorkerSpec(DQSG, 3, 5, seed=worker_seed(6, 0)), WorkerSpec(NDQSG, 2, 0, 4, 2.0, 1.0, worker_seed(6, 1)),
+             WorkerSpec(NDQSG, 2, 0, 4, 2.0, 1.0, worker_seed(6, 2))]
+    grads = [(c + 0.003 * rng.standard_normal(n)).astype(np.float32) for _ in specs]
+    omsgs, gmsgs, _keep = _messages(dq, oracle, specs, grads, bucket, step)
+    host_msgs = [dq.Message(torch.from_numpy(om.packed.view(np.int32).copy()).pin_memory(),
+                            torch.from_numpy(om.scale.copy()).pin_memory(), sp.seed, w, sp.kind, gm.params)
+                 for w, (om, gm, sp) in enumerate(zip(omsgs, gmsgs, specs))]
+    ws = torch.empty(dq.decode_workspace_bytes(host_msgs, n, False), dtype=torch.uint8, device="cuda")
+    out = host_output(torch, n, torch.float32)
+    dq.ndqsg_decode_aggregate_side_first_host(host_msgs, n, step, out, ws)
+    dev = dq.ndqsg_decode_aggregate_side_first(gmsgs, n, step)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.numpy().view(np.uint32), dev[:n].cpu().numpy().view(np.uint32))
