@@ -270,18 +270,22 @@ class GpuState:
         return enc, dec
 
 
-def time_isolated(torch, launches, iters=24, warm=3):
-    """Average duration (ms) of the launches in `launches` (callables on rotating buffers), CUDA events."""
+def time_isolated(torch, launches, iters=24, warm=3, repeats=3):
+    """Average duration (ms) of the launches in `launches` (callables on rotating buffers) between two CUDA
+    events; the median of `repeats` such averages."""
     for i in range(warm):
         launches[i % len(launches)]()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(iters):
-        launches[i % len(launches)]()
-    e1.record()
-    torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / iters
+    avgs = []
+    for _ in range(repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            launches[i % len(launches)]()
+        e1.record()
+        torch.cuda.synchronize()
+        avgs.append(e0.elapsed_time(e1) / iters)
+    return statistics.median(avgs)
 
 
 def kernel_timings(st: GpuState, hbm_peak, sm_max_mhz):

@@ -270,7 +270,8 @@ dq_status encode_common(dq_kind kind, const float* grad, uint64_t n, uint64_t se
         tile_ctas = (uint32_t)(want_ctas < room ? want_ctas : room);
     }
     // the spacing only pays when the first requests of all resident warps saturate HBM
-    a.request_spacing_ns = (uint32_t)((uint64_t)dq::kFirstRequestSpacingNs * tile_ctas / slots);
+    // (a launch that reads early gets its CTAs one by one, as the previous kernel's CTAs leave: nothing to space)
+    a.request_spacing_ns = a.early_read ? 0u : (uint32_t)((uint64_t)dq::kFirstRequestSpacingNs * tile_ctas / slots);
     const bool d16 = (p->dither_bits == 16u);
     if (launch_encode(mode, p->bits, d16, map, a, plain + tile_ctas, st) != cudaSuccess) return DQ_ERR_CUDA;
     g_launches.fetch_add(1);

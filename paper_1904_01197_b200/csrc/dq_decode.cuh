@@ -417,7 +417,9 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
             float v[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                v[e] = (args.invW != 0.0f) ? __fmul_rn(acc[4 * c + e], args.invW) : __fdiv_rn(acc[4 * c + e], args.Wf);
+                v[e] = (args.W == 1u)        ? acc[4 * c + e]                       // the mean of one message is itself
+                       : (args.invW != 0.0f) ? __fmul_rn(acc[4 * c + e], args.invW)
+                                             : __fdiv_rn(acc[4 * c + e], args.Wf);
             asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
                          ::"r"(row_addr ^ (uint32_t)(c << 4)), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3])
                          : "memory");
