@@ -1,4 +1,5 @@
-"""Bandwidth sweep of the encode and fused decode-aggregate kernels (BASELINE config 5).
+"""Bandwidth sweep of the encode and fused decode-aggregate kernels: n from 2^16 to 2^28, W in {2, 8, 32}, 1-4
+bits, buckets of 256 to 8192 elements.
 
     python -m bench_tools.sweep [--quick] [--out FILE]
 

@@ -76,10 +76,13 @@ struct DecodeArgs {
     DecWorker w[64];
 };
 
-constexpr int kDecThreads = 128;
+#ifndef DQ_DEC_THREADS
+#define DQ_DEC_THREADS 128
+#endif
+constexpr int kDecThreads = DQ_DEC_THREADS;
 constexpr int kDecWarps = kDecThreads / 32;
 #ifndef DQ_DEC_MINBLOCKS
-#define DQ_DEC_MINBLOCKS 4
+#define DQ_DEC_MINBLOCKS (512 / DQ_DEC_THREADS)
 #endif
 constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;     // resident CTAs per SM the register budget is set for
 constexpr int kDecTileBytes = 32 * 128;         // one unit of side information or output
@@ -317,8 +320,12 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
 
     const uint32_t total_warps = gridDim.x * (uint32_t)kDecWarps;
     const uint32_t gw = blockIdx.x * (uint32_t)kDecWarps + warp;
-    if (gw >= args.num_units) return;
-    const uint32_t my_units = (args.num_units - gw - 1u) / total_warps + 1u;
+    // units of this warp, and of the CTA's first warp (which has the most): the warps of a CTA take four adjacent
+    // units at a time and meet before each, so that they run through the same code at about the same time and
+    // share its instruction-cache lines
+    const uint32_t my_units = (gw < args.num_units) ? (args.num_units - gw - 1u) / total_warps + 1u : 0u;
+    const uint32_t cta_gw = blockIdx.x * (uint32_t)kDecWarps;
+    const uint32_t cta_units = (cta_gw < args.num_units) ? (args.num_units - cta_gw - 1u) / total_warps + 1u : 0u;
     const uint32_t whole_rows = args.full_rows - args.first_row;       // rows of the tile maps
 
     // side information of this warp's k-th unit -> tile buffer k mod 3 (lane 0)
@@ -340,7 +347,7 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
             for (uint32_t l = 0; l < lines; ++l) prefetch_l2(p + 32u * l);
         }
     };
-    if (lane == 0 && side_tiles) issue_side(0u);
+    if (lane == 0 && side_tiles && my_units != 0u) issue_side(0u);
     __syncwarp();
 
     // bucket of a row (rows past the end take the last row's bucket: their results are never stored)
@@ -355,7 +362,9 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
     float kappa_next = __ldg(args.w[0].scale + bucket);
 
 #pragma unroll 1
-    for (uint32_t k = 0; k < my_units; ++k) {
+    for (uint32_t k = 0; k < cta_units; ++k) {
+        __syncthreads();
+        if (k >= my_units) continue;
         const uint32_t unit = gw + k * total_warps;
         const uint32_t row = args.first_row + unit * 32u + lane;
         const uint32_t b = k % (uint32_t)kDecTileBuffers;

@@ -1,4 +1,5 @@
-"""GPU parity at the full BASELINE sizes, in the launch configuration bench.py times: the whole vector goes
+"""GPU parity at the full workload sizes (11.7 M, 25.6 M and 124 M elements; 4 M-element sweep points), in the
+launch configuration bench.py times: the whole vector goes
 through the CUDA library; the oracle recomputes sampled bucket ranges (it can handle any bucket range on its
 own because the dither counter uses the index in the whole gradient) and every sampled word, scale and output
 value is compared.  Nothing the oracle consumes comes from the CUDA path."""
