@@ -728,7 +728,8 @@ def main():
             roofline_decode = {"kernel": dec_name, "bound": "alu", "achieved": alg_instr / kd["ms"] / 1e9,
                                "peak": alu_peak / 1e12, "unit": "Tlane-instr/s",
                                "frac": alg_instr / kd["ms"] * 1e3 / alu_peak,
-                               "traffic": kernels["decode_aggregate"].get("traffic") if dec_name == "decode_aggregate" else None,
+                               "traffic": (committed_counters().get(f"{cfg.name}.{dec_name}.dram_bytes")
+                                           if dith == 32 else None),
                                "peak_source": "148 SMs x 4 schedulers x 32 lanes x max SM clock",
                                "hbm_gbs": kd["gbs"], "frac_hbm": kd["frac_hbm"], "launches_per_step": 1,
                                "gelem_worker_s": kd["gelem_worker_s"],
