@@ -329,6 +329,9 @@ dq_status decode_common(const dq_msg* msgs, uint32_t W, uint64_t n, uint64_t ste
         }
         d.variant = kind * 8u + m.p.bits - 1u;
     }
+    // runs of equal variants (one routine per run, see decode_workers)
+    for (uint32_t w = W; w-- > 0u;)
+        a.w[w].group_end = (w + 1u < W && a.w[w + 1u].variant == a.w[w].variant) ? a.w[w + 1u].group_end : w + 1u;
     if (first_element % msgs[0].p.bucket != 0u) return DQ_ERR_INVALID_ARG;   // a range starts at a bucket boundary
     if (n == 0) return DQ_OK;
     if (n >= (1ull << 34) || first_element >= (1ull << 34) || first_element + n >= (1ull << 34))

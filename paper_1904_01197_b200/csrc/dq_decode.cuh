@@ -34,6 +34,7 @@ struct DecWorker {
     const uint32_t* packed;   // } addresses of the (virtual) whole-gradient buffers, see DecodeArgs
     const float* scale;       // }
     uint32_t unit_lines;      // 128-byte lines of one unit's packed words (= bits)
+    uint32_t group_end;       // index after the last worker of the run of equal variants that this worker belongs to
     PhiloxStream ps;
     uint32_t variant;     // DecKind * 8 + bits - 1: one jump selects the routine
     uint32_t bits;
@@ -204,25 +205,60 @@ __device__ __forceinline__ void decode_row(const DecWorker& wk, uint32_t row, ui
     }
 }
 
-// Dispatch on (kind, bits): one indexed jump.
-template <int DITH, bool RUN>
-__device__ __forceinline__ void decode_row_variant(const DecWorker& wk, uint32_t row, uint32_t load_row,
-                                                   float kappa, uint32_t side_addr, float (&acc)[32],
-                                                   uint32_t bias_bits)
+// State of a lane while it walks over the workers of a unit.
+struct DecLane {
+    uint32_t row, load_row, bucket, bucket_next, row_addr, kappa_bits_max;
+    float kappa_next;
+};
+
+// The workers [w, w_end) of one run of equal variants: the same routine for each, so the jump on the variant is taken
+// once per run and not once per worker (Algorithm 2's groups P1 and P2 are two runs).
+template <int BITS, uint32_t KIND, int DITH, int SIDE>
+__device__ __forceinline__ void decode_run(const DecodeArgs& args, uint32_t w, uint32_t w_end, DecLane& ln, float (&acc)[32])
+{
+#pragma unroll 1
+    for (; w < w_end; ++w) {
+        const float kappa = ln.kappa_next;
+        // the next step's scale: the next worker's for this bucket, or the first worker's for the next unit
+        ln.kappa_next = (w + 1u < args.W) ? __ldg(args.w[w + 1u].scale + ln.bucket)
+                                          : __ldg(args.w[0].scale + ln.bucket_next);
+        decode_row<BITS, KIND, DITH, SIDE == kSideRunning>(args.w[w], ln.row, ln.load_row, kappa, ln.row_addr, acc,
+                                                            args.half_bias_bits);
+        if (SIDE == kSideFirst && w == 0u) {
+            // the accumulators are now the reconstruction of message 0: it is the side information of the nested
+            // messages that follow, which read it from the lane's row of the tile buffer
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
+                             ::"r"(ln.row_addr ^ (uint32_t)(c << 4)), "f"(acc[4 * c]), "f"(acc[4 * c + 1]),
+                               "f"(acc[4 * c + 2]), "f"(acc[4 * c + 3])
+                             : "memory");
+        }
+        const uint32_t kb = __float_as_uint(kappa) & 0x7FFFFFFFu;
+        ln.kappa_bits_max = (kb > ln.kappa_bits_max) ? kb : ln.kappa_bits_max;
+    }
+}
+
+// All W workers of a unit, run by run; dispatch on (kind, bits) with one jump per run.
+template <int DITH, int SIDE>
+__device__ __forceinline__ void decode_workers(const DecodeArgs& args, DecLane& ln, float (&acc)[32])
 {
 #define DQ_DEC_CASE(KIND, BITS)                                                                                    \
-    case (KIND) * 8u + (BITS) - 1u:                                                                                \
-        decode_row<BITS, KIND, DITH, RUN>(wk, row, load_row, kappa, side_addr, acc, bias_bits);                        \
-        break;
+    case (KIND) * 8u + (BITS) - 1u: decode_run<BITS, KIND, DITH, SIDE>(args, w, w_end, ln, acc); break;
 #define DQ_DEC_KIND(KIND)                                                                                          \
     DQ_DEC_CASE(KIND, 1) DQ_DEC_CASE(KIND, 2) DQ_DEC_CASE(KIND, 3) DQ_DEC_CASE(KIND, 4)                            \
     DQ_DEC_CASE(KIND, 5) DQ_DEC_CASE(KIND, 6) DQ_DEC_CASE(KIND, 7) DQ_DEC_CASE(KIND, 8)
-    switch (wk.variant) {
-        DQ_DEC_KIND(kDecDqsg)
-        DQ_DEC_KIND(kDecNdqsgPow2)
-        DQ_DEC_KIND(kDecNdqsgPow2Shrink)
-        DQ_DEC_KIND(kDecNdqsgAnyK)
-        default: break;
+#pragma unroll 1
+    for (uint32_t w = 0; w < args.W;) {
+        const uint32_t w_end = args.w[w].group_end;
+        switch (args.w[w].variant) {
+            DQ_DEC_KIND(kDecDqsg)
+            DQ_DEC_KIND(kDecNdqsgPow2)
+            DQ_DEC_KIND(kDecNdqsgPow2Shrink)
+            DQ_DEC_KIND(kDecNdqsgAnyK)
+            default: break;
+        }
+        w = w_end;
     }
 #undef DQ_DEC_KIND
 #undef DQ_DEC_CASE
@@ -392,32 +428,16 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
         float acc[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
-        uint32_t kappa_bits_max = 0u;
-
+        DecLane ln;
+        ln.row = row; ln.load_row = load_row; ln.bucket = bucket; ln.bucket_next = bucket_next;
+        ln.row_addr = row_addr; ln.kappa_bits_max = 0u; ln.kappa_next = kappa_next;
         if (unit_has_tile) {
-#pragma unroll 1
-            for (uint32_t w = 0; w < args.W; ++w) {
-                const float kappa = kappa_next;
-                // the next step's scale: the next worker's for this bucket, or the first worker's for the next unit
-                kappa_next = (w + 1u < args.W) ? __ldg(args.w[w + 1u].scale + bucket)
-                                               : __ldg(args.w[0].scale + bucket_next);
-                decode_row_variant<DITH, RUN>(args.w[w], row, load_row, kappa, row_addr, acc, args.half_bias_bits);
-                if (SIDE == kSideFirst && w == 0u) {
-                    // the accumulators are now the reconstruction of message 0: it is the side information of
-                    // the nested messages that follow, which read it from the lane's row of the tile buffer
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
-                                     ::"r"(row_addr ^ (uint32_t)(c << 4)), "f"(acc[4 * c]), "f"(acc[4 * c + 1]),
-                                       "f"(acc[4 * c + 2]), "f"(acc[4 * c + 3])
-                                     : "memory");
-                }
-                const uint32_t kb = __float_as_uint(kappa) & 0x7FFFFFFFu;
-                kappa_bits_max = (kb > kappa_bits_max) ? kb : kappa_bits_max;
-            }
+            decode_workers<DITH, SIDE>(args, ln, acc);
+            kappa_next = ln.kappa_next;
         } else {
             kappa_next = __ldg(args.w[0].scale + bucket_next);
         }
+        const uint32_t kappa_bits_max = ln.kappa_bits_max;
         bucket = bucket_next;
 
         // the mean leaves through the tile buffer: the lane writes its row where it read its side information
