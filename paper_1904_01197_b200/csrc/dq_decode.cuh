@@ -2,8 +2,11 @@
 // server loop with the side information given as a vector or taken as the running mean).
 //
 // One lane owns one row = 32 consecutive elements: 32 fp32 accumulators in registers, and per worker exactly
-// `bits` packed words.  A warp owns a unit of 32 rows and is autonomous: persistent warps take units round-robin
-// and never wait for one another.
+// `bits` packed words.  A warp owns a unit of 32 rows.  One persistent CTA of sixteen warps runs per SM; its
+// warps form teams of four that take four adjacent units at a time from the CTA's share of the gradient.  The
+// share is fixed (CTA c owns every gridDim.x-th group of four units), the order inside it is not: teams draw the
+// next group from a counter in shared memory, because the warp schedulers favour some warps by a fifth and a
+// fixed split would leave the favoured ones idle at the end.
 //   * The side information of a unit arrives in the warp's shared memory by one 2-D tile copy (32 rows x 128
 //     bytes, 128-byte swizzle, so that "lane r reads row r" is free of bank conflicts), issued one unit ahead.
 //   * Every worker's packed words of the next unit are requested into the L2 one unit ahead (one prefetch
@@ -78,7 +81,7 @@ struct DecodeArgs {
 };
 
 #ifndef DQ_DEC_THREADS
-#define DQ_DEC_THREADS 128
+#define DQ_DEC_THREADS 512
 #endif
 constexpr int kDecThreads = DQ_DEC_THREADS;
 constexpr int kDecWarps = kDecThreads / 32;
@@ -86,6 +89,13 @@ constexpr int kDecWarps = kDecThreads / 32;
 #define DQ_DEC_MINBLOCKS (512 / DQ_DEC_THREADS)
 #endif
 constexpr int kDecMinBlocks = DQ_DEC_MINBLOCKS;     // resident CTAs per SM the register budget is set for
+#ifndef DQ_DEC_TEAM
+#define DQ_DEC_TEAM 4
+#endif
+constexpr int kDecTeamWarps = DQ_DEC_TEAM;          // warps that take adjacent units and meet before each
+constexpr int kDecTeams = kDecWarps / kDecTeamWarps;
+static_assert(kDecWarps % kDecTeamWarps == 0 && kDecTeams >= 1 && (kDecTeamWarps == 1 || kDecTeams <= 15),
+              "teams of several warps use named barriers 1..15");
 constexpr int kDecTileBytes = 32 * 128;         // one unit of side information or output
 constexpr int kDecTileBuffers = 3;              // per warp: side in flight / side in use, then output leaving
 // Dynamic shared memory of a CTA: the warps' tile buffers (plus room to align to 1024 bytes).
@@ -264,13 +274,15 @@ __device__ __forceinline__ void decode_workers(const DecodeArgs& args, DecLane& 
 #undef DQ_DEC_CASE
 }
 
-// The last row of a gradient whose length is not a multiple of 32: one element at a time, everything at run
-// time, straight from and to global memory.  Same arithmetic, in the same order, as decode_row.
+// The last row of a gradient whose length is not a multiple of 32: one element per lane (`e` = the lane, of a
+// whole warp), everything at run time, straight from and to global memory.  Same arithmetic, in the same order,
+// as decode_row.  Each element is a chain of dependent loads and divisions, about a microsecond per worker.
 template <int DITH, int SIDE>
-__device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint32_t row, uint32_t bucket, uint32_t nvalid)
+__device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint32_t row, uint32_t bucket, uint32_t nvalid,
+                                                uint32_t e)
 {
     constexpr bool RUN = (SIDE == kSideRunning);
-    for (uint32_t e = 0; e < nvalid; ++e) {
+    if (e < nvalid) {
         const uint64_t i = (uint64_t)row * 32u + e;
         float yside = (!RUN && args.has_side) ? __ldg(args.side + i) : 0.0f;
         float acc = 0.0f;
@@ -322,7 +334,8 @@ __device__ __noinline__ void decode_partial_row(const DecodeArgs& args, uint32_t
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The decode kernel.  Grid = persistent CTAs of four autonomous warps; dynamic shared memory = kDecSmemBytes.
+// The decode kernel.  Grid = persistent CTAs (one per SM) of teams of four warps; dynamic shared memory =
+// kDecSmemBytes.
 // side_map / out_map: [whole rows x 32 floats] views of the caller's side information and output (valid when
 // args.use_tiles; side_map only when args.has_side).
 // ---------------------------------------------------------------------------------------------------
@@ -331,7 +344,6 @@ __global__ void __launch_bounds__(kDecThreads, kDecMinBlocks)
 decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __grid_constant__ CUtensorMap out_map,
                         const __grid_constant__ DecodeArgs args)
 {
-    constexpr bool RUN = (SIDE == kSideRunning);
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_side_mem[kDecWarps][kDecTileBuffers];
 
@@ -354,23 +366,38 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
     // the messages (and the side information) may be the previous kernel's output
     grid_dependency_wait();
 
-    const uint32_t total_warps = gridDim.x * (uint32_t)kDecWarps;
-    const uint32_t gw = blockIdx.x * (uint32_t)kDecWarps + warp;
-    // units of this warp, and of the CTA's first warp (which has the most): the warps of a CTA take four adjacent
-    // units at a time and meet before each, so that they run through the same code at about the same time and
-    // share its instruction-cache lines
-    const uint32_t my_units = (gw < args.num_units) ? (args.num_units - gw - 1u) / total_warps + 1u : 0u;
-    const uint32_t cta_gw = blockIdx.x * (uint32_t)kDecWarps;
-    const uint32_t cta_units = (cta_gw < args.num_units) ? (args.num_units - cta_gw - 1u) / total_warps + 1u : 0u;
+    // Work: a team-unit is kDecTeamWarps adjacent units (32 rows each), one per warp of a team.  CTA c owns the
+    // team-units c, c + gridDim.x, ...; its teams draw them from a counter in shared memory, one ahead of the
+    // one they work on, so a team that the schedulers favour simply takes more of them and all teams of an SM
+    // finish within one unit of each other.  The warps of a team meet before each unit: they run through the
+    // same code at about the same time and share its instruction-cache lines.
+    __shared__ uint32_t draw_count;
+    __shared__ uint32_t drawn[kDecTeams][2];
+    const uint32_t team = warp / (uint32_t)kDecTeamWarps;
+    const uint32_t tw = warp % (uint32_t)kDecTeamWarps;
+    const uint32_t num_tunits = (args.num_units + (uint32_t)kDecTeamWarps - 1u) / (uint32_t)kDecTeamWarps;
+    const uint32_t cta_tunits = (blockIdx.x < num_tunits) ? (num_tunits - blockIdx.x - 1u) / gridDim.x + 1u : 0u;
+    auto team_meet = [&]() {
+        if constexpr (kDecTeams == 1) __syncthreads();
+        else if constexpr (kDecTeamWarps == 1) __syncwarp();
+        else asm volatile("bar.sync %0, %1;" ::"r"(team + 1u), "n"(kDecTeamWarps * 32) : "memory");
+    };
+    // unit of this warp in the CTA's j-th team-unit (>= num_units: none)
+    auto unit_of = [&](uint32_t j) {
+        return (j < cta_tunits) ? (blockIdx.x + j * gridDim.x) * (uint32_t)kDecTeamWarps + tw : 0xFFFFFFFFu;
+    };
+    if (threadIdx.x == 0) draw_count = 0u;
+    __syncthreads();
+    if (tw == 0u && lane == 0u) drawn[team][0] = atomicAdd(&draw_count, 1u);
+    team_meet();
+    uint32_t unit = unit_of(drawn[team][0]);
     const uint32_t whole_rows = args.full_rows - args.first_row;       // rows of the tile maps
 
-    // side information of this warp's k-th unit -> tile buffer k mod 3 (lane 0)
-    auto issue_side = [&](uint32_t k) {
-        if ((gw + k * total_warps) * 32u >= whole_rows) return;         // a unit that is only the ragged last row
-        const uint32_t b = k % (uint32_t)kDecTileBuffers;
+    // side information of unit `u` -> tile buffer `b` (lane 0)
+    auto issue_side = [&](uint32_t u, uint32_t b) {
+        if (u * 32u >= whole_rows) return;                              // a unit that is only the ragged last row
         mbar_expect_tx(bar_side + 8u * b, (uint32_t)kDecTileBytes);
-        tma_load_rows(tiles + b * (uint32_t)kDecTileBytes, &side_map, bar_side + 8u * b,
-                      (int32_t)((gw + k * total_warps) * 32u));
+        tma_load_rows(tiles + b * (uint32_t)kDecTileBytes, &side_map, bar_side + 8u * b, (int32_t)(u * 32u));
     };
     // Ask the L2 for every worker's packed words of the unit that starts at row `row0`: lane w (and w + 32)
     // requests the 128-byte lines of worker w, whose words of a unit are 128 * bits contiguous bytes.
@@ -383,7 +410,7 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
             for (uint32_t l = 0; l < lines; ++l) prefetch_l2(p + 32u * l);
         }
     };
-    if (lane == 0 && side_tiles && my_units != 0u) issue_side(0u);
+    if (lane == 0 && side_tiles && unit < args.num_units) issue_side(unit, 0u);
     __syncwarp();
 
     // bucket of a row (rows past the end take the last row's bucket: their results are never stored)
@@ -392,32 +419,40 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
         return (args.rpb_shift != 0xFFFFFFFFu) ? (rc >> args.rpb_shift) : (rc / args.rows_per_bucket);
     };
 
+    // The ragged last row goes first, on the warp that tends to have the least to do: left to the end of the
+    // unit that contains it, its serial chains would be what the whole grid waits for.
+    if (args.full_rows < args.rows && blockIdx.x == gridDim.x - 1u && warp == (uint32_t)kDecWarps - 1u)
+        decode_partial_row<DITH, SIDE>(args, args.full_rows, bucket_of(args.full_rows),
+                                       (uint32_t)(args.n - (uint64_t)args.full_rows * 32u), lane);
+
     const uint32_t swz16 = (lane & 7u) << 4;
     bool gave_up = false;
-    uint32_t bucket = bucket_of(args.first_row + gw * 32u + lane);
+    uint32_t bucket = bucket_of(args.first_row + (unit < args.num_units ? unit : 0u) * 32u + lane);
     float kappa_next = __ldg(args.w[0].scale + bucket);
 
 #pragma unroll 1
-    for (uint32_t k = 0; k < cta_units; ++k) {
-        __syncthreads();
-        if (k >= my_units) continue;
-        const uint32_t unit = gw + k * total_warps;
+    for (uint32_t it = 0; unit != 0xFFFFFFFFu; ++it) {
+        // draw the next team-unit, then meet: everyone has read the previous draw before the one after this
+        if (tw == 0u && lane == 0u) drawn[team][(it + 1u) & 1u] = atomicAdd(&draw_count, 1u);
+        team_meet();
+        const uint32_t unit_next = unit_of(drawn[team][(it + 1u) & 1u]);
+        if (unit >= args.num_units) { unit = unit_next; continue; }    // past the end (last team-unit only)
         const uint32_t row = args.first_row + unit * 32u + lane;
-        const uint32_t b = k % (uint32_t)kDecTileBuffers;
+        const uint32_t b = it % (uint32_t)kDecTileBuffers;
         const uint32_t tile = tiles + b * (uint32_t)kDecTileBytes;
-        const bool more = k + 1u < my_units;
-        const uint32_t bucket_next = more ? bucket_of(row + total_warps * 32u) : bucket;
-        if (more) prefetch_words(row - lane + total_warps * 32u);
+        const bool more = unit_next < args.num_units;
+        const uint32_t bucket_next = more ? bucket_of(args.first_row + unit_next * 32u + lane) : bucket;
+        if (more) prefetch_words(args.first_row + unit_next * 32u);
         if (lane == 0) {
             // the store issued two units ago has read its buffer: that buffer takes the next unit's side
             // information now and this unit's output later
             bulk_wait_group_read<1>();
-            if (side_tiles && more) issue_side(k + 1u);
+            if (side_tiles && more) issue_side(unit_next, (it + 1u) % (uint32_t)kDecTileBuffers);
         }
         __syncwarp();
         const bool unit_has_tile = unit * 32u < whole_rows;
         if (side_tiles && unit_has_tile &&
-            !mbar_wait_bounded(bar_side + 8u * b, (k / (uint32_t)kDecTileBuffers) & 1u, gave_up)) {
+            !mbar_wait_bounded(bar_side + 8u * b, (it / (uint32_t)kDecTileBuffers) & 1u, gave_up)) {
             gave_up = true;
             if (lane == 0) atomicOr(args.error_flags, 0x2u);
         }
@@ -460,8 +495,7 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
             bulk_commit_group();
         }
         if (args.status != nullptr && kappa_bits_max >= 0x7F800000u && row < args.full_rows) atomicOr(args.status, 0x1u);
-        if (row == args.full_rows && row < args.rows)
-            decode_partial_row<DITH, SIDE>(args, row, bucket_of(row), (uint32_t)(args.n - (uint64_t)row * 32u));
+        unit = unit_next;
     }
     // shared memory must stay valid until the last stores have read it
     if (lane == 0) bulk_wait_group_read<0>();

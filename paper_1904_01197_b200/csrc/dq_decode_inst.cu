@@ -35,7 +35,7 @@ cudaError_t DQ_NAME(DQ_INST_DITH, DQ_INST_RUN)(const CUtensorMap& side_map, cons
     }
     const uint32_t smem = kDecSmemBytes;
     const int blocks = per_sm[dev].load();
-    const uint64_t want = ((uint64_t)a.num_units + kDecWarps - 1u) / kDecWarps;
+    const uint64_t want = ((uint64_t)a.num_units + kDecTeamWarps - 1u) / kDecTeamWarps;   // one team-unit each at least
     const uint64_t room = (uint64_t)blocks * (uint64_t)sm_count;
     const uint32_t grid = (uint32_t)(want < room ? want : room);
     return launch_overlapped(k, grid, (uint32_t)kDecThreads, smem, st, side_map, out_map, a);
