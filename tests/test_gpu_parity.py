@@ -183,6 +183,51 @@ def test_decode_ragged_lengths(dq, oracle, n):
         assert_fp32_close(got, ref, f"n={n} bucket={bucket}")
 
 
+@pytest.mark.parametrize("units", [1, 3, 4, 5, 9, 147, 148, 149, 591, 592, 593, 597, 1187])
+def test_decode_unit_counts(dq, oracle, units):
+    """Lengths around the decoder's work distribution: a unit is 32 rows of 32 elements, warps take units in
+    teams of four and a CTA per SM draws its teams' units from a counter, so the counts that matter are multiples
+    of 4 and of (4 x number of SMs) and their neighbours; each with a whole last row, a ragged one and a short
+    last unit."""
+    rng = np.random.default_rng(650 + units)
+    bucket = 2048
+    for short in (0, 1, 1000):
+        n = units * 1024 - short
+        side = rng.standard_normal(n).astype(np.float32)
+        grads = [(side + 0.05 * rng.standard_normal(n)).astype(np.float32) for _ in range(2)]
+        specs = [WorkerSpec(DQSG, 3, 5, seed=43), WorkerSpec(NDQSG, 2, 0, 4, 2.0, 1.0, 44)]
+        got, ref = _roundtrip_decode(dq, oracle, 2, n, bucket, specs, grads, side, step=9)
+        assert assert_fp32_close(got, ref, f"units={units} n={n}")
+
+
+def test_decode_with_a_wrong_step_matches_the_oracles_wrong_decode(dq, oracle):
+    """A message whose header is corrupt (here: decoded at another step than it was encoded at) cannot be detected
+    from the codes; the decoder must then compute exactly what the definition gives for that step, dither of the
+    wrong stream and all, and must not flag the scales."""
+    rng = np.random.default_rng(660)
+    n, bucket, W, step = 9 * 2048 + 333, 2048, 3, 11
+    side = rng.standard_normal(n).astype(np.float32)
+    grads = [(side + 0.05 * rng.standard_normal(n)).astype(np.float32) for _ in range(W)]
+    specs = [WorkerSpec(DQSG, 3, 5, seed=45), WorkerSpec(NDQSG, 2, 0, 4, 2.0, 1.0, 46),
+             WorkerSpec(NDQSG, 3, 0, 6, 9.0, 0.9, 47)]
+    omsgs, gmsgs, keep = [], [], []
+    for w in range(W):
+        opk, osc = oracle_encode(oracle, grads[w], specs[w], w, step, bucket)
+        omsgs.append(oracle_msg(oracle, opk, osc, specs[w], w, bucket))
+        pk = torch.from_numpy(np.concatenate([opk, np.zeros(4, np.uint32)]).view(np.int32)).cuda()
+        sc = torch.from_numpy(osc.copy()).cuda()
+        keep.append((pk, sc))
+        gmsgs.append(gpu_msg(dq, pk, sc, specs[w], w, bucket))
+    right = oracle.decode_aggregate(omsgs, n, step, side_info=side, threads=4)
+    wrong = oracle.decode_aggregate(omsgs, n, step + 1, side_info=side, threads=4)
+    assert np.abs(wrong - right).max() > 0.01                 # the other stream's dither is visible
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    out = dq.ndqsg_decode_aggregate(gmsgs, n, step + 1, torch.from_numpy(side).cuda(), status_word=status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    assert assert_fp32_close(out[:n].cpu().numpy(), wrong, "wrong step")
+
+
 def test_decode_dqsg_only_and_shrinkage(dq, oracle):
     rng = np.random.default_rng(700)
     n, bucket, W = 50_000, 2048, 4

@@ -139,6 +139,26 @@ def test_dqsg_unbiased_over_iterations():
     assert abs(z.mean()) < 5 / math.sqrt(n)
 
 
+def test_dqsg_decoded_with_another_dither_stream_triples_the_error():
+    """A message decoded with the wrong seed or step (a corrupt header): the receiver subtracts a dither u' that is
+    independent of the sender's u, so the error in units of Delta is e + u - u' with e, u, u' independent and
+    uniform on (-1/2, 1/2): variance 3/12 instead of 1/12, and no longer bounded by 1/2.  (Schuchman's condition,
+    Section 3.1: only the SAME dither makes the error independent of the signal.)"""
+    rng = np.random.default_rng(31)
+    n, B, levels = 1 << 17, 1024, 15
+    g = (rng.standard_normal(n) * 0.01).astype(np.float32)
+    packed, scale, _ = oracle.dqsg_encode(g, SEED, 1, 3, B, 4, levels, want_codes=True)
+    kappa = np.repeat(scale.astype(np.float64), B)[:n]
+    Delta = 2.0 / (levels - 1)
+    for seed, worker, step in ((SEED + 1, 1, 3), (SEED, 2, 3), (SEED, 1, 4)):
+        msg = oracle.Msg(packed, scale, seed, worker, oracle.KIND_DQSG, B, 4, levels)
+        rec = oracle.decode_aggregate([msg], n, step)
+        e = (rec.astype(np.float64) - g.astype(np.float64)) / kappa / Delta
+        assert abs(e.var() - 3 / 12) < 0.03 * (3 / 12), (seed, worker, step, e.var())
+        assert np.abs(e).max() > 1.0                                            # up to 3/2, never above
+        assert np.abs(e).max() <= 1.5 + 1e-5
+
+
 # ------------------------------------------------------------------ Appendix A: selection probabilities
 @pytest.mark.parametrize("M,x", [(1, 0.3), (2, 0.3), (2, -0.7), (3, 0.95)])
 def test_level_selection_probabilities(M, x):
