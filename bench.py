@@ -738,6 +738,13 @@ def main():
                                                    "pipe_cycles_per_wide_multiply": 4.0,
                                                    "floor_cycles_per_element_worker": 4.0 * wide_per_unit,
                                                    "frac": 4.0 * wide_per_unit / cyc_per_unit}}
+            probe = (other or {}).get("issue_probe", {})
+            if dith == 32 and "decode_mix_ceiling_gelem_worker_s" in probe:
+                # what the decoder's arithmetic alone (nine rounds for four blocks, then 16 NDQSG elements) reaches
+                # on this GPU, measured in this run by bench_tools/issue_probe
+                roofline_decode["measured_mix_ceiling"] = {
+                    "gelem_worker_s": probe["decode_mix_ceiling_gelem_worker_s"],
+                    "frac": kd["gelem_worker_s"] / probe["decode_mix_ceiling_gelem_worker_s"]}
             if kd["ms"] >= count[dom_enc] * ke["ms"]:
                 roofline = roofline_decode
             else:
