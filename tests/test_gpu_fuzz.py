@@ -100,3 +100,48 @@ def test_random_host_buffer_round_trip(dq, oracle, case):
     ref = oracle.decode_aggregate(omsgs, n, step, side_info=side if any_nd else None, threads=4)
     assert_fp32_close(out.numpy(), ref, f"case {case}")
     assert dq.device_error_flags() == 0
+
+
+@pytest.mark.parametrize("case", range(15))
+def test_random_decode_with_several_draws_per_cta(dq, oracle, case):
+    """Lengths up to three million elements, where every persistent decoder CTA draws several groups of units, in
+    the three side-information modes (a given vector, the reconstruction of message 0, the running mean)."""
+    from dq_testlib import gpu_msg, oracle_encode, oracle_msg
+    rng = np.random.default_rng(910_000 + case)
+    bucket = int(rng.choice(BUCKETS))
+    n = int(rng.integers(1, 3_000_000))
+    if case % 5 == 0:
+        n = max(1024, (n // 1024) * 1024)                          # whole units now and then
+    W = int(rng.integers(1, 10))
+    dither_bits = 16 if case % 3 == 2 else 32
+    step = int(rng.integers(0, 2 ** 40))
+    mode = case % 3
+    c = rng.standard_normal(n).astype(np.float32)
+    grads = [(c + 0.2 * rng.standard_normal(n)).astype(np.float32) for _ in range(W)]
+    specs = [_random_spec(rng, dither_bits) for _ in range(W)]
+    if mode != 0:                                                  # Algorithm 2: the first message is DQSG
+        specs[0] = WorkerSpec(DQSG, 3, int(rng.integers(2, 9)), seed=int(rng.integers(0, 2 ** 63)),
+                              dither_bits=dither_bits)
+    omsgs, gmsgs, keep = [], [], []
+    for w, (sp, g) in enumerate(zip(specs, grads)):
+        opk, osc = oracle_encode(oracle, g, sp, w, step, bucket)
+        omsgs.append(oracle_msg(oracle, opk, osc, sp, w, bucket))
+        pk = torch.from_numpy(np.concatenate([opk, np.zeros(4, np.uint32)]).view(np.int32)).cuda()
+        sc = torch.from_numpy(osc.copy()).cuda()
+        keep.append((pk, sc))
+        gmsgs.append(gpu_msg(dq, pk, sc, sp, w, bucket))
+    any_nd = any(s.kind == NDQSG for s in specs)
+    if mode == 0:
+        ref = oracle.decode_aggregate(omsgs, n, step, side_info=c if any_nd else None, threads=8)
+        out = (dq.ndqsg_decode_aggregate(gmsgs, n, step, torch.from_numpy(c).cuda()) if any_nd
+               else dq.dqsg_decode_aggregate(gmsgs, n, step))
+    elif mode == 1:
+        side = oracle.decode_aggregate(omsgs[:1], n, step, threads=8)
+        ref = oracle.decode_aggregate(omsgs, n, step, side_info=side, threads=8)
+        out = dq.ndqsg_decode_aggregate_side_first(gmsgs, n, step)
+    else:
+        ref = oracle.decode_aggregate(omsgs, n, step, running=True, threads=8)
+        out = dq.ndqsg_decode_aggregate_running(gmsgs, n, step)
+    torch.cuda.synchronize()
+    assert_fp32_close(out[:n].cpu().numpy(), ref, f"case {case}: mode={mode} bucket={bucket} n={n} specs={specs}")
+    assert dq.device_error_flags() == 0
