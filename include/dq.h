@@ -95,6 +95,9 @@ typedef struct {
  * Then nothing in the encoder waits for that kernel except its own end: the two kernels overlap wherever the
  * GPU has room (the tail of one runs beside the head of the next), while a later kernel that waits for this
  * one still sees both complete.  Results are identical with and without the flag.
+ * "Neither reads nor writes" is about the memory, not the pointer: a buffer that a stream-ordered allocator
+ * hands out may be memory that the previous kernel still reads (its input, freed by the host a moment ago);
+ * such a buffer is not free in this sense.
  */
 #define DQ_FLAG_OUTPUT_FREE 0x2u
 /*

@@ -83,6 +83,24 @@ def _run_full_size(dq, oracle, cfg, seed=0):
         out = dq.dqsg_decode_aggregate(gmsgs, n, step)
     torch.cuda.synchronize()
     out_h = out[:n].cpu().numpy()
+    if cfg.side_from_worker0:
+        # the launch configuration of the benchmark step: every encode with the early-read / early-store launch
+        # flags, back to back, then the fused decode that takes its side information from message 0
+        flagged, live = [], []        # the gradients stay allocated: a freed one could be handed out as an output
+        for w, spec in enumerate(cfg.workers):
+            p = spec_params(dq, spec, B)
+            p.flags = dq.DQ_FLAG_INPUT_READY | (dq.DQ_FLAG_OUTPUT_FREE if w > 0 else 0)
+            live.append(torch.from_numpy(cfg.grad(w)).cuda())
+            fn = dq.dqsg_encode if spec.kind == DQSG else dq.ndqsg_encode
+            flagged.append(fn(live[-1], spec.seed, w, step, p))
+        fused = dq.ndqsg_decode_aggregate_side_first([gpu_msg(dq, pk, sc, spec, w, B) for w, (spec, (pk, sc))
+                                                      in enumerate(zip(cfg.workers, flagged))], n, step)
+        torch.cuda.synchronize()
+        for w, ((pk, sc), (pk0, sc0)) in enumerate(zip(flagged, keep)):
+            assert torch.equal(pk, pk0) and torch.equal(sc, sc0), f"worker {w}: the launch flags changed the message"
+        assert np.array_equal(fused[:n].cpu().numpy().view(np.uint32), out_h.view(np.uint32)), \
+            "the fused side information changed the result"
+        del flagged, fused, live
     exact = True
     for (b0, b1) in ranges:
         lo, hi = b0 * B, min(n, b1 * B)
