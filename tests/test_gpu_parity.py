@@ -29,7 +29,7 @@ def oracle():
 
 
 from dq_testlib import (assert_fp32_close, gpu_encode, gpu_msg, host_output, oracle_encode, oracle_msg,  # noqa: E402
-                        words_np)
+                        spec_params, words_np)
 
 
 def _specs_for_bits(bits):
@@ -226,6 +226,42 @@ def test_decode_with_a_wrong_step_matches_the_oracles_wrong_decode(dq, oracle):
     torch.cuda.synchronize()
     assert int(status[0]) == 0
     assert assert_fp32_close(out[:n].cpu().numpy(), wrong, "wrong step")
+
+
+def test_decodes_and_encodes_on_two_streams_at_once(dq, oracle):
+    """Launches of the library that run side by side on two streams share nothing but the error word: results are
+    those of the same calls made one after the other."""
+    rng = np.random.default_rng(670)
+    n, bucket, step, W = 1_500_000 + 77, 2048, 4, 4
+    jobs = []
+    for j in range(2):
+        side = rng.standard_normal(n).astype(np.float32)
+        grads = [(side + 0.05 * rng.standard_normal(n)).astype(np.float32) for _ in range(W)]
+        specs = [WorkerSpec(DQSG, 3, 5, seed=100 + j)] + [WorkerSpec(NDQSG, 2, 0, 4, 2.0, 1.0, 110 + 10 * j + w)
+                                                         for w in range(1, W)]
+        gdev = [torch.from_numpy(g).cuda() for g in grads]
+        jobs.append((specs, gdev, torch.from_numpy(side).cuda()))
+    def run(j, stream):
+        specs, gdev, side = jobs[j]
+        msgs = []
+        for w, sp in enumerate(specs):
+            p = spec_params(dq, sp, bucket)
+            fn = dq.dqsg_encode if sp.kind == DQSG else dq.ndqsg_encode
+            pk, sc = fn(gdev[w], sp.seed, w, step, p, stream=stream)
+            msgs.append(gpu_msg(dq, pk, sc, sp, w, bucket))
+        return msgs, dq.ndqsg_decode_aggregate(msgs, n, step, side, stream=stream)
+    torch.cuda.synchronize()
+    serial = [run(j, None) for j in range(2)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for rep in range(3):
+        both = [run(j, streams[j]) for j in range(2)]
+        torch.cuda.synchronize()
+        for j in range(2):
+            for m_s, m_b in zip(serial[j][0], both[j][0]):
+                assert torch.equal(m_s.packed, m_b.packed) and torch.equal(m_s.scale, m_b.scale)
+            assert torch.equal(serial[j][1], both[j][1]), f"job {j}, repetition {rep}"
+    assert dq.device_error_flags() == 0
 
 
 def test_decode_dqsg_only_and_shrinkage(dq, oracle):
