@@ -1,5 +1,6 @@
 // Fused decode-and-average kernel (Algorithm 1, server steps; nested decoder equation and Algorithm 2,
-// server loop with the side information given as a vector or taken as the running mean).
+// server loop with the side information given as a vector, taken as the running mean, or taken as the
+// reconstruction of message 0).
 //
 // One lane owns one row = 32 consecutive elements: 32 fp32 accumulators in registers, and per worker exactly
 // `bits` packed words.  A warp owns a unit of 32 rows.  One persistent CTA of sixteen warps runs per SM; its
@@ -369,8 +370,8 @@ decode_aggregate_kernel(const __grid_constant__ CUtensorMap side_map, const __gr
     // Work: a team-unit is kDecTeamWarps adjacent units (32 rows each), one per warp of a team.  CTA c owns the
     // team-units c, c + gridDim.x, ...; its teams draw them from a counter in shared memory, one ahead of the
     // one they work on, so a team that the schedulers favour simply takes more of them and all teams of an SM
-    // finish within one unit of each other.  The warps of a team meet before each unit: they run through the
-    // same code at about the same time and share its instruction-cache lines.
+    // finish within one unit of each other.  The warps of a team meet before each unit, so that they run through
+    // the same code at about the same time (teams of one to four warps measure alike, larger ones are slower).
     __shared__ uint32_t draw_count;
     __shared__ uint32_t drawn[kDecTeams][2];
     const uint32_t team = warp / (uint32_t)kDecTeamWarps;
